@@ -1,0 +1,146 @@
+/* fp2 -- block-sparse causal prefill attention for B200 (sm_100a): C ABI.
+ *
+ * Two stages (Algorithm 1 of the paper):
+ *   stage 1  fp2_select_blocks   block-mean pooling (Eq. 5), block energies of every (KV head, packed query
+ *                                tile, KV block) (Eq. 19), max-based threshold plus forced sink / window /
+ *                                diagonal blocks (Eq. 3, Eq. 20) -> per-(sequence, KV head, tile) block lists;
+ *   stage 2  fp2_sparse_prefill  flash attention over the listed blocks, the unlisted fully visible blocks
+ *                                entering through their pooled means (mean correction, Eq. 6), over a paged
+ *                                KV cache (Eq. 22) in a continuous batch with PackGQA row packing (Eq. 13).
+ *   fp2_dense_prefill is stage 2 with every candidate block attended exactly.
+ *
+ * Conventions common to all calls
+ *   - Every tensor pointer is a DEVICE pointer unless its name starts with h_ (host).  The caller owns all
+ *     tensors, list buffers and the workspace; the library owns only the plan object.  Stage calls allocate
+ *     and free nothing, enqueue their kernels on the given stream and return without synchronising.
+ *   - Layouts (row-major, innermost last):
+ *       q, out        [total_q, num_q_heads, 128]        BF16 (out always BF16; q BF16 or FP8 e4m3)
+ *       k_cache, v_cache [num_pages, page_size, num_kv_heads, 128]   BF16 or FP8 e4m3
+ *       page_table    int32 [num_seqs, max_pages_per_seq]; token j of sequence b lives in slot
+ *                     page_table[b][j / page_size] * page_size + j % page_size  (Eq. 22)
+ *       cu_seqlens_q  int32 [num_seqs + 1]  offsets of the sequences' new tokens in q / out
+ *       seqlens_k     int32 [num_seqs]      total KV tokens (cached prefix + new tokens)
+ *       q_scale [num_q_heads], k_scale / v_scale [num_kv_heads]  fp32 de-quantisation scales, FP8 only
+ *                     (NULL for BF16); per-tensor scaling (Eq. 15) is the case of equal entries
+ *       lse           fp32 [num_q_heads, total_q], natural log of the softmax denominator (may be NULL)
+ *     Query i of sequence b sits at absolute position (seqlens_k[b] - Lq_b) + i: the causal mask is aligned
+ *     to the end of the KV sequence, so cached prefixes (chunked prefill) are visible to every new token.
+ *   - Segments.  With g = num_q_heads / num_kv_heads, packed row r of a KV head's query matrix is position
+ *     r / g, query head h_kv * g + r % g (Eq. 13); tile t holds packed rows [128 t, 128 (t+1)).  Segment
+ *     seg = num_kv_heads * tile_off[b] + h_kv * ntiles_b + t, ntiles_b = ceil(g * Lq_b / 128), tile_off the
+ *     exclusive scan of ntiles.  Lists are a padded CSR: seg_offset[seg] (fixed by the plan: exclusive scan
+ *     of the candidate counts J_hi + 1), seg_count[seg] selected blocks, blk_idx[seg_offset[seg] + k]
+ *     ascending ids of 128-token KV blocks.
+ *   - Errors.  Every call returns an fp2_status.  Problems visible on the host (null pointers, unsupported
+ *     shapes, lengths that disagree with the plan) are reported before anything is launched.  The device
+ *     never traps: waits inside the kernels are bounded and list entries are clamped; both conditions are
+ *     recorded in a status block that fp2_read_status returns.
+ */
+#ifndef FP2_H_
+#define FP2_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FP2_OK = 0,
+  FP2_ERR_INVALID_ARG = 1,  /* null pointer, inconsistent lengths, malformed list seen on the device */
+  FP2_ERR_UNSUPPORTED = 2,  /* head_dim != 128, block_size != 128, page_size not dividing 128, ...    */
+  FP2_ERR_CAPACITY = 3,     /* sequence longer than the compiled maximum                              */
+  FP2_ERR_CUDA = 4,         /* a CUDA runtime / driver call failed                                    */
+  FP2_ERR_TIMEOUT = 5       /* a bounded wait inside a kernel expired                                 */
+} fp2_status;
+
+typedef enum { FP2_BF16 = 0, FP2_FP8_E4M3 = 1 } fp2_dtype;
+
+typedef struct fp2_plan fp2_plan; /* opaque */
+typedef void* fp2_stream;         /* a cudaStream_t passed as an address-sized handle; NULL = default */
+
+/* Shapes and method parameters (Sec. 4.1: B = 128, 256 sink tokens, 512-token window, alpha = 0.1). */
+typedef struct {
+  int32_t num_seqs, total_q, num_q_heads, num_kv_heads;
+  int32_t head_dim;       /* must be 128                                                              */
+  int32_t block_size;     /* B, KV tokens per selection block; must be 128                            */
+  int32_t tile_rows;      /* packed query rows per tile; must be 128                                  */
+  int32_t page_size;      /* p; 8, 16, 32, 64 or 128                                                  */
+  int32_t num_pages, max_pages_per_seq;
+  int32_t sink_tokens;    /* blocks J < ceil(sink_tokens / B) are always selected                     */
+  int32_t window_tokens;  /* blocks J >= J_lo - ceil(window_tokens / B) are always selected           */
+  int32_t use_correction; /* 1: Eq. 6 (mean correction); 0: Eq. 4 (plain truncation)                  */
+  float alpha;            /* threshold factor of Eq. 3 / Eq. 20                                       */
+  float softmax_scale;    /* 0 selects 1 / sqrt(head_dim)                                             */
+  int32_t dtype;          /* fp2_dtype of q, k_cache, v_cache                                         */
+} fp2_params;
+
+/* Planner (host side; the per-step metadata of Sec. 3.4 "Serving Integration").  Takes HOST copies of the
+ * lengths, builds the segment table and uploads it to the current device (one small allocation owned by the
+ * plan, freed by fp2_plan_destroy).  h_cu_seqlens_q has num_seqs + 1 entries, h_seqlens_k num_seqs.
+ * Returns FP2_ERR_INVALID_ARG for null / inconsistent input (Lq_b < 0, Lq_b > Lk_b, sum Lq != total_q, pages
+ * needed > max_pages_per_seq), FP2_ERR_UNSUPPORTED / FP2_ERR_CAPACITY for shapes outside the compiled
+ * kernels (see fp2_status).  *out is written only on FP2_OK.  If no CUDA device is usable the plan is still
+ * returned -- sizes and the segment table can be queried -- but stage calls on it return FP2_ERR_CUDA. */
+fp2_status fp2_plan_create(const fp2_params* params, const int32_t* h_cu_seqlens_q, const int32_t* h_seqlens_k,
+                           fp2_plan** out);
+
+/* Sizes the caller needs: number of segments, capacity of blk_idx in entries (worst case = all candidate
+ * pairs), bytes of device workspace (pooled statistics, work order, status block).  Any output may be NULL. */
+fp2_status fp2_plan_sizes(const fp2_plan* plan, int64_t* num_segments, int64_t* idx_capacity,
+                          int64_t* workspace_bytes);
+
+void fp2_plan_destroy(fp2_plan* plan);
+
+/* Host-side view of one row of the segment table (PackGQA geometry, Eq. 13; candidates 0..J_hi):
+ * out10 = {b, h_kv, t, first packed row, real rows, prefix length, Lk, J_lo, J_hi, first pooled-block row of
+ * the sequence}; *list_offset = seg_offset[seg] (may be NULL).  Host memory; needs no device. */
+fp2_status fp2_plan_segment(const fp2_plan* plan, int64_t seg, int32_t* out10, int64_t* list_offset);
+
+/* Stage 1 (Algorithm 1, lines 1-5).  Pools K and V into per-block means kept in `workspace`, scores every
+ * candidate block of every segment and writes the lists.
+ *   out: seg_offset int64 [num_segments + 1], seg_count int32 [num_segments], blk_idx int32 [idx_capacity].
+ * v_cache is read here because the pooled V means (used by stage 2's correction) are produced in the same
+ * pass.  The workspace must be at least workspace_bytes and 1024-byte aligned, and must be passed unchanged to
+ * the following fp2_sparse_prefill.  Its first 128 bytes hold the status block and the work counter and
+ * must be zero before the first stage call (fp2_read_status clears the status block again). */
+fp2_status fp2_select_blocks(fp2_plan* plan, const void* q, const void* k_cache, const void* v_cache,
+                             const int32_t* page_table, const int32_t* cu_seqlens_q, const int32_t* seqlens_k,
+                             const float* q_scale, const float* k_scale, const float* v_scale,
+                             int64_t* seg_offset, int32_t* seg_count, int32_t* blk_idx, void* workspace,
+                             fp2_stream stream);
+
+/* Stage 2 (Algorithm 1, lines 6-11; Eq. 4, Eq. 6).  Attends exactly over the listed blocks; with
+ * use_correction = 1 every unlisted block J < J_lo (fully visible to the whole tile) contributes
+ * |B_J| e^{q.kbar_J / sqrt(d)} (vbar_J, 1) to numerator and denominator.  The lists may come from
+ * fp2_select_blocks or from the caller (ascending, unique, within 0..J_hi; entries outside are clamped and
+ * flagged in the status block).  `pooled_valid` != 0 says the workspace still holds the pooled means of a
+ * preceding fp2_select_blocks on the same inputs; 0 makes this call recompute them.
+ *   out: out BF16 [total_q, num_q_heads, 128]; lse fp32 [num_q_heads, total_q] or NULL. */
+fp2_status fp2_sparse_prefill(fp2_plan* plan, const void* q, const void* k_cache, const void* v_cache,
+                              const int32_t* page_table, const int32_t* cu_seqlens_q, const int32_t* seqlens_k,
+                              const int64_t* seg_offset, const int32_t* seg_count, const int32_t* blk_idx,
+                              const float* q_scale, const float* k_scale, const float* v_scale, void* out,
+                              float* lse, void* workspace, int32_t pooled_valid, fp2_stream stream);
+
+/* Dense causal attention through the same kernel: every candidate block 0..J_hi of every tile is attended
+ * exactly, nothing is pooled or corrected (the paper's own dense baseline, Sec. 3.3). */
+fp2_status fp2_dense_prefill(fp2_plan* plan, const void* q, const void* k_cache, const void* v_cache,
+                             const int32_t* page_table, const int32_t* cu_seqlens_q, const int32_t* seqlens_k,
+                             const float* q_scale, const float* k_scale, const float* v_scale, void* out,
+                             float* lse, void* workspace, fp2_stream stream);
+
+/* Synchronises `stream`, reads the status block of `workspace` and clears it.  Returns FP2_ERR_TIMEOUT if a
+ * bounded wait expired, FP2_ERR_INVALID_ARG if a list entry had to be clamped, else FP2_OK.  If
+ * h_status_words is not NULL it receives the 8 raw int32 words (host memory). */
+fp2_status fp2_read_status(fp2_plan* plan, void* workspace, int32_t* h_status_words, fp2_stream stream);
+
+/* Number of kernels the last stage call on this plan enqueued (host counter). */
+int32_t fp2_last_launch_count(const fp2_plan* plan);
+
+const char* fp2_status_string(fp2_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FP2_H_ */

@@ -1,0 +1,400 @@
+// C ABI of the library (declared in include/fp2.h): host-side planner, argument checks, TMA tensor maps,
+// kernel launches.  No device memory is allocated in the stage calls; the plan owns one small device table.
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "../../include/fp2.h"
+#include "common.cuh"
+#include "pool_kv.cuh"
+#include "score_select.cuh"
+#include "sparse_attn.cuh"
+
+using namespace fp2;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct fp2_plan {
+  fp2_params prm;
+  DevParams dev;
+  int device;
+  int num_sms;
+  int64_t nseg, idx_capacity, nblk_tot;
+  std::vector<int32_t> h_cu_q, h_lk;
+  std::vector<SegInfo> h_segs;
+  // device table owned by the plan: [SegInfo x nseg][blk_off x (ns+1)]
+  void* d_table;
+  SegInfo* d_segs;
+  int32_t* d_blk_off;
+  // workspace layout (byte offsets)
+  int64_t ws_status, ws_counter, ws_khi, ws_klo, ws_vbar, ws_order, ws_hist, ws_bytes;
+  EncodeTiledFn encode;
+  int32_t last_launches;
+  bool attrs_set;
+};
+
+static inline int64_t align_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+extern "C" const char* fp2_status_string(fp2_status s) {
+  switch (s) {
+    case FP2_OK: return "ok";
+    case FP2_ERR_INVALID_ARG: return "invalid argument";
+    case FP2_ERR_UNSUPPORTED: return "unsupported shape or dtype";
+    case FP2_ERR_CAPACITY: return "sequence exceeds compiled capacity";
+    case FP2_ERR_CUDA: return "CUDA error";
+    case FP2_ERR_TIMEOUT: return "bounded wait expired inside a kernel";
+  }
+  return "unknown status";
+}
+
+extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, const int32_t* h_lk, fp2_plan** out) {
+  if (!p || !h_cu || !h_lk || !out) return FP2_ERR_INVALID_ARG;
+  if (p->num_seqs <= 0 || p->total_q < 0 || p->num_q_heads <= 0 || p->num_kv_heads <= 0) return FP2_ERR_INVALID_ARG;
+  if (p->num_q_heads % p->num_kv_heads != 0) return FP2_ERR_INVALID_ARG;
+  if (p->head_dim != kHeadDim || p->block_size != kBlock || p->tile_rows != kTileRows) return FP2_ERR_UNSUPPORTED;
+  const int ps = p->page_size;
+  if (!(ps == 8 || ps == 16 || ps == 32 || ps == 64 || ps == 128)) return FP2_ERR_UNSUPPORTED;
+  if (p->dtype != FP2_BF16 && p->dtype != FP2_FP8_E4M3) return FP2_ERR_UNSUPPORTED;
+  if (p->num_pages <= 0 || p->max_pages_per_seq <= 0) return FP2_ERR_INVALID_ARG;
+  if (p->sink_tokens < 0 || p->window_tokens < 0) return FP2_ERR_INVALID_ARG;
+  if (!(p->alpha == p->alpha) || p->softmax_scale < 0.f) return FP2_ERR_INVALID_ARG;
+  if (h_cu[0] != 0 || h_cu[p->num_seqs] != p->total_q) return FP2_ERR_INVALID_ARG;
+
+  const int g = p->num_q_heads / p->num_kv_heads;
+  int64_t ntiles_tot = 0, nblk_tot = 0;
+  for (int b = 0; b < p->num_seqs; ++b) {
+    const int64_t lq = (int64_t)h_cu[b + 1] - h_cu[b], lk = h_lk[b];
+    if (lq < 0 || lk < 0 || lq > lk) return FP2_ERR_INVALID_ARG;
+    if ((lk + ps - 1) / ps > p->max_pages_per_seq) return FP2_ERR_INVALID_ARG;
+    const int64_t nblk = (lk + kBlock - 1) / kBlock;
+    if (nblk > kMaxBlocks) return FP2_ERR_CAPACITY;
+    ntiles_tot += (g * lq + kTileRows - 1) / kTileRows;
+    nblk_tot += nblk;
+  }
+  if (ntiles_tot * p->num_kv_heads > (int64_t)0x7fffffff || nblk_tot > (int64_t)0x7fffffff) return FP2_ERR_CAPACITY;
+
+  fp2_plan* pl = new (std::nothrow) fp2_plan();
+  if (!pl) return FP2_ERR_CUDA;
+  pl->prm = *p;
+  pl->h_cu_q.assign(h_cu, h_cu + p->num_seqs + 1);
+  pl->h_lk.assign(h_lk, h_lk + p->num_seqs);
+  pl->nseg = ntiles_tot * p->num_kv_heads;
+  pl->nblk_tot = nblk_tot;
+  pl->d_table = nullptr;
+  pl->last_launches = 0;
+  pl->attrs_set = false;
+
+  // segment table: seg = Hkv * tile_off[b] + h * ntiles_b + t
+  std::vector<SegInfo> segs((size_t)pl->nseg);
+  std::vector<int32_t> blk_off((size_t)p->num_seqs + 1);
+  int64_t tile_off = 0, off = 0, boff = 0;
+  for (int b = 0; b < p->num_seqs; ++b) {
+    const int lq = h_cu[b + 1] - h_cu[b], lk = h_lk[b], pre = lk - lq;
+    const int nt = (int)(((int64_t)g * lq + kTileRows - 1) / kTileRows);
+    blk_off[b] = (int32_t)boff;
+    for (int h = 0; h < p->num_kv_heads; ++h)
+      for (int t = 0; t < nt; ++t) {
+        SegInfo& s = segs[(size_t)(p->num_kv_heads * tile_off + (int64_t)h * nt + t)];
+        const int64_t r0 = (int64_t)t * kTileRows;
+        const int64_t r1 = r0 + kTileRows < (int64_t)g * lq ? r0 + kTileRows : (int64_t)g * lq;
+        s.b = b; s.h = h; s.t = t;
+        s.nrows = (int)(r1 - r0);
+        s.q_tok0 = h_cu[b];
+        s.r0 = (int)r0;
+        s.pre = pre;
+        s.Lk = lk;
+        s.J_lo = (int)((pre + r0 / g) / kBlock);
+        s.J_hi = (int)((pre + (r1 - 1) / g) / kBlock);
+        s.blk_off = (int32_t)boff;
+        s.pad = 0;
+        s.off = 0;
+      }
+    tile_off += nt;
+    boff += (lk + kBlock - 1) / kBlock;
+  }
+  blk_off[p->num_seqs] = (int32_t)boff;
+  for (int64_t i = 0; i < pl->nseg; ++i) {
+    segs[(size_t)i].off = off;
+    off += segs[(size_t)i].J_hi + 1;
+  }
+  pl->idx_capacity = off;
+
+  // Device part.  Without a usable CUDA device the plan is still returned (sizes and the segment table can be
+  // queried), but every stage call on it fails with FP2_ERR_CUDA.
+  pl->device = -1;
+  pl->num_sms = 0;
+  pl->encode = nullptr;
+  cudaDeviceProp prop;
+  int dev = -1;
+  if (cudaGetDevice(&dev) == cudaSuccess && cudaGetDeviceProperties(&prop, dev) == cudaSuccess) {
+    if (prop.major != 10) { delete pl; return FP2_ERR_UNSUPPORTED; }
+    pl->device = dev;
+    pl->num_sms = prop.multiProcessorCount;
+    const size_t seg_bytes = (size_t)align_up((int64_t)sizeof(SegInfo) * (pl->nseg > 0 ? pl->nseg : 1), 256);
+    const size_t tab_bytes = seg_bytes + sizeof(int32_t) * blk_off.size();
+    if (cudaMalloc(&pl->d_table, tab_bytes) != cudaSuccess) { delete pl; return FP2_ERR_CUDA; }
+    pl->d_segs = reinterpret_cast<SegInfo*>(pl->d_table);
+    pl->d_blk_off = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(pl->d_table) + seg_bytes);
+    if ((pl->nseg > 0 && cudaMemcpy(pl->d_segs, segs.data(), sizeof(SegInfo) * segs.size(),
+                                    cudaMemcpyHostToDevice) != cudaSuccess) ||
+        cudaMemcpy(pl->d_blk_off, blk_off.data(), sizeof(int32_t) * blk_off.size(), cudaMemcpyHostToDevice) !=
+            cudaSuccess) {
+      cudaFree(pl->d_table);
+      delete pl;
+      return FP2_ERR_CUDA;
+    }
+    cudaDriverEntryPointQueryResult qres;
+    void* fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) {
+      cudaFree(pl->d_table);
+      delete pl;
+      return FP2_ERR_CUDA;
+    }
+    pl->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  } else {
+    (void)cudaGetLastError();
+  }
+  pl->h_segs.swap(segs);
+
+  // workspace layout
+  const int64_t pooled = align_up(nblk_tot * p->num_kv_heads * kHeadDim * 2, 1024);
+  int64_t o = 0;
+  pl->ws_status = o;  o += 64;
+  pl->ws_counter = o; o += 64;
+  o = align_up(o, 1024);
+  pl->ws_khi = o;  o += pooled;
+  pl->ws_klo = o;  o += pooled;
+  pl->ws_vbar = o; o += pooled;
+  pl->ws_order = o; o += align_up(4 * (pl->nseg > 0 ? pl->nseg : 1), 1024);
+  pl->ws_hist = o;  o += align_up(4 * ((int64_t)p->num_kv_heads * kCountBuckets + 1), 1024);
+  pl->ws_bytes = o;
+
+  DevParams& d = pl->dev;
+  d.num_q_heads = p->num_q_heads; d.num_kv_heads = p->num_kv_heads; d.group = g;
+  d.page_size = ps; d.pages_per_block = kBlock / ps; d.max_pages_per_seq = p->max_pages_per_seq;
+  d.num_pages = p->num_pages;
+  d.sink_blocks = (p->sink_tokens + kBlock - 1) / kBlock;
+  d.window_blocks = (p->window_tokens + kBlock - 1) / kBlock;
+  d.use_correction = p->use_correction ? 1 : 0;
+  d.num_seqs = p->num_seqs; d.nseg = (int32_t)pl->nseg; d.nblk_tot = (int32_t)nblk_tot; d.total_q = p->total_q;
+  d.fp8 = p->dtype == FP2_FP8_E4M3;
+  d.alpha = p->alpha;
+  const double sc = p->softmax_scale > 0.f ? (double)p->softmax_scale : 1.0 / sqrt((double)kHeadDim);
+  d.scale_log2 = (float)(sc * 1.4426950408889634);
+  *out = pl;
+  return FP2_OK;
+}
+
+extern "C" fp2_status fp2_plan_sizes(const fp2_plan* pl, int64_t* nseg, int64_t* cap, int64_t* ws) {
+  if (!pl) return FP2_ERR_INVALID_ARG;
+  if (nseg) *nseg = pl->nseg;
+  if (cap) *cap = pl->idx_capacity;
+  if (ws) *ws = pl->ws_bytes;
+  return FP2_OK;
+}
+
+extern "C" void fp2_plan_destroy(fp2_plan* pl) {
+  if (!pl) return;
+  if (pl->d_table) cudaFree(pl->d_table);
+  delete pl;
+}
+
+extern "C" fp2_status fp2_plan_segment(const fp2_plan* pl, int64_t seg, int32_t* out10, int64_t* list_offset) {
+  if (!pl || !out10 || seg < 0 || seg >= pl->nseg) return FP2_ERR_INVALID_ARG;
+  const SegInfo& s = pl->h_segs[(size_t)seg];
+  const int32_t v[10] = {s.b, s.h, s.t, s.r0, s.nrows, s.pre, s.Lk, s.J_lo, s.J_hi, s.blk_off};
+  memcpy(out10, v, sizeof(v));
+  if (list_offset) *list_offset = s.off;
+  return FP2_OK;
+}
+
+extern "C" int32_t fp2_last_launch_count(const fp2_plan* pl) { return pl ? pl->last_launches : 0; }
+
+// ------------------------------------------------------------------------------------------------------
+// helpers
+// ------------------------------------------------------------------------------------------------------
+// 3-D map over [rows, heads, 128] elements, box = [box_rows, 1, 64 (bf16) | 128 (fp8)], 128-byte swizzle.
+static bool make_map(fp2_plan* pl, CUtensorMap* m, const void* base, int64_t rows, int heads, int box_rows, bool fp8) {
+  const int esz = fp8 ? 1 : 2;
+  cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)heads, (cuuint64_t)rows};
+  cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * esz, (cuuint64_t)kHeadDim * esz * heads};
+  cuuint32_t box[3] = {(cuuint32_t)(128 / esz), 1u, (cuuint32_t)box_rows};
+  cuuint32_t es[3] = {1, 1, 1};
+  CUresult r = pl->encode(m, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                          const_cast<void*>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+static fp2_status set_attrs(fp2_plan* pl) {
+  if (pl->attrs_set) return FP2_OK;
+  if (cudaFuncSetAttribute(score_select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kScoreSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(score_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kScoreSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(sparse_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kAttnSmemBytes) != cudaSuccess)
+    return FP2_ERR_CUDA;
+  pl->attrs_set = true;
+  return FP2_OK;
+}
+
+static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+static fp2_status check_common(fp2_plan* pl, const void* q, const void* k, const void* v, const int32_t* pt,
+                               const int32_t* cu, const int32_t* lk, const float* qs, const float* ks,
+                               const float* vs, const void* ws) {
+  if (!pl || !q || !k || !v || !pt || !cu || !lk || !ws) return FP2_ERR_INVALID_ARG;
+  if (pl->dev.fp8 && (!qs || !ks || !vs)) return FP2_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(ws, 1024)) return FP2_ERR_INVALID_ARG;
+  if (pl->device < 0) return FP2_ERR_CUDA;  // plan was made without a device
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FP2_ERR_CUDA;
+  if (dev != pl->device) return FP2_ERR_INVALID_ARG;
+  return set_attrs(pl);
+}
+
+static fp2_status launch_pool(fp2_plan* pl, const void* k, const void* v, const int32_t* pt, const int32_t* lk,
+                              const float* ks, const float* vs, uint8_t* ws, cudaStream_t st) {
+  if (pl->nblk_tot == 0) return FP2_OK;
+  dim3 grid((unsigned)pl->nblk_tot, (unsigned)pl->prm.num_kv_heads);
+  __nv_bfloat16* khi = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_khi);
+  __nv_bfloat16* klo = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_klo);
+  __nv_bfloat16* vb = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_vbar);
+  if (pl->dev.fp8)
+    pool_kv_kernel<true><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, lk, pl->d_blk_off, ks, vs,
+                                               pl->dev, khi, klo, vb);
+  else
+    pool_kv_kernel<false><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, lk, pl->d_blk_off, ks, vs,
+                                                pl->dev, khi, klo, vb);
+  pl->last_launches += 1;
+  return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
+}
+
+// counting sort of the segments: KV-head-major, descending block count
+static fp2_status launch_order(fp2_plan* pl, const int32_t* seg_count, uint8_t* ws, cudaStream_t st) {
+  const int nseg = (int)pl->nseg;
+  int32_t* hist = reinterpret_cast<int32_t*>(ws + pl->ws_hist);
+  int32_t* order = reinterpret_cast<int32_t*>(ws + pl->ws_order);
+  const int nb = pl->prm.num_kv_heads * kCountBuckets;
+  if (cudaMemsetAsync(hist, 0, sizeof(int32_t) * (size_t)(nb + 1), st) != cudaSuccess) return FP2_ERR_CUDA;
+  if (cudaMemsetAsync(ws + pl->ws_counter, 0, 64, st) != cudaSuccess) return FP2_ERR_CUDA;
+  const int blocks = (nseg + 255) / 256;
+  order_hist_kernel<<<blocks, 256, 0, st>>>(pl->d_segs, seg_count, nseg, hist);
+  order_scan_kernel<<<1, 1024, 0, st>>>(hist, nb);
+  order_scatter_kernel<<<blocks, 256, 0, st>>>(pl->d_segs, seg_count, nseg, hist, order);
+  pl->last_launches += 3;
+  return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// stage 1
+// ------------------------------------------------------------------------------------------------------
+extern "C" fp2_status fp2_select_blocks(fp2_plan* pl, const void* q, const void* k, const void* v, const int32_t* pt,
+                                        const int32_t* cu, const int32_t* lk, const float* qs, const float* ks,
+                                        const float* vs, int64_t* seg_offset, int32_t* seg_count, int32_t* blk_idx,
+                                        void* workspace, fp2_stream stream) {
+  fp2_status s = check_common(pl, q, k, v, pt, cu, lk, qs, ks, vs, workspace);
+  if (s != FP2_OK) return s;
+  if (!seg_offset || !seg_count || !blk_idx) return FP2_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  pl->last_launches = 0;
+  if (pl->nseg == 0) return FP2_OK;
+  if ((s = launch_pool(pl, k, v, pt, lk, ks, vs, ws, st)) != FP2_OK) return s;
+  CUtensorMap mhi, mlo;
+  if (!make_map(pl, &mhi, ws + pl->ws_khi, pl->nblk_tot, pl->prm.num_kv_heads, 128, false) ||
+      !make_map(pl, &mlo, ws + pl->ws_klo, pl->nblk_tot, pl->prm.num_kv_heads, 128, false))
+    return FP2_ERR_CUDA;
+  int* status = reinterpret_cast<int*>(ws + pl->ws_status);
+  if (pl->dev.fp8)
+    score_select_kernel<true><<<(unsigned)pl->nseg, kScoreThreads, kScoreSmemBytes, st>>>(
+        mhi, mlo, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, status);
+  else
+    score_select_kernel<false><<<(unsigned)pl->nseg, kScoreThreads, kScoreSmemBytes, st>>>(
+        mhi, mlo, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, status);
+  pl->last_launches += 1;
+  return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// stage 2 (sparse and dense)
+// ------------------------------------------------------------------------------------------------------
+static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, const void* v, const int32_t* pt,
+                                const int32_t* cu, const int32_t* lk, const int32_t* seg_count,
+                                const int32_t* blk_idx, const float* qs, const float* ks, const float* vs, void* out,
+                                float* lse, void* workspace, bool need_pool, fp2_stream stream) {
+  fp2_status s = check_common(pl, q, k, v, pt, cu, lk, qs, ks, vs, workspace);
+  if (s != FP2_OK) return s;
+  if (!out || !aligned(out, 16)) return FP2_ERR_INVALID_ARG;
+  if (pl->dev.fp8) return FP2_ERR_UNSUPPORTED;  // FP8 attention kernel not built yet
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  pl->last_launches = 0;
+  if (pl->nseg == 0) return FP2_OK;
+  if (need_pool && (s = launch_pool(pl, k, v, pt, lk, ks, vs, ws, st)) != FP2_OK) return s;
+  if ((s = launch_order(pl, seg_count, ws, st)) != FP2_OK) return s;
+  const bool fp8 = pl->dev.fp8 != 0;
+  const int64_t slots = (int64_t)pl->prm.num_pages * pl->prm.page_size;
+  CUtensorMap mk, mv, mkb, mvb;
+  if (!make_map(pl, &mk, k, slots, pl->prm.num_kv_heads, pl->prm.page_size, fp8) ||
+      !make_map(pl, &mv, v, slots, pl->prm.num_kv_heads, pl->prm.page_size, fp8) ||
+      !make_map(pl, &mkb, ws + pl->ws_khi, pl->nblk_tot, pl->prm.num_kv_heads, 128, false) ||
+      !make_map(pl, &mvb, ws + pl->ws_vbar, pl->nblk_tot, pl->prm.num_kv_heads, 128, false))
+    return FP2_ERR_CUDA;
+  AttnArgs a;
+  a.q = reinterpret_cast<const uint8_t*>(q);
+  a.page_table = pt;
+  a.segs = pl->d_segs;
+  a.order = reinterpret_cast<const int32_t*>(ws + pl->ws_order);
+  a.seg_count = seg_count;
+  a.blk_idx = blk_idx;
+  a.q_scale = qs; a.k_scale = ks; a.v_scale = vs;
+  a.out = reinterpret_cast<__nv_bfloat16*>(out);
+  a.lse = lse;
+  a.work_counter = reinterpret_cast<int*>(ws + pl->ws_counter);
+  a.status = reinterpret_cast<int*>(ws + pl->ws_status);
+  const unsigned grid = (unsigned)(pl->nseg < pl->num_sms ? pl->nseg : pl->num_sms);
+  sparse_attn_kernel<false><<<grid, kAttnThreads, kAttnSmemBytes, st>>>(mk, mv, mkb, mvb, a, pl->dev);
+  pl->last_launches += 1;
+  return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
+}
+
+extern "C" fp2_status fp2_sparse_prefill(fp2_plan* pl, const void* q, const void* k, const void* v,
+                                         const int32_t* pt, const int32_t* cu, const int32_t* lk,
+                                         const int64_t* seg_offset, const int32_t* seg_count, const int32_t* blk_idx,
+                                         const float* qs, const float* ks, const float* vs, void* out, float* lse,
+                                         void* workspace, int32_t pooled_valid, fp2_stream stream) {
+  if (!seg_offset || !seg_count || !blk_idx) return FP2_ERR_INVALID_ARG;
+  const bool need_pool = pl && pl->dev.use_correction && !pooled_valid;
+  return run_attention(pl, q, k, v, pt, cu, lk, seg_count, blk_idx, qs, ks, vs, out, lse, workspace, need_pool,
+                       stream);
+}
+
+extern "C" fp2_status fp2_dense_prefill(fp2_plan* pl, const void* q, const void* k, const void* v, const int32_t* pt,
+                                        const int32_t* cu, const int32_t* lk, const float* qs, const float* ks,
+                                        const float* vs, void* out, float* lse, void* workspace, fp2_stream stream) {
+  return run_attention(pl, q, k, v, pt, cu, lk, nullptr, nullptr, qs, ks, vs, out, lse, workspace, false, stream);
+}
+
+extern "C" fp2_status fp2_read_status(fp2_plan* pl, void* workspace, int32_t* h_words, fp2_stream stream) {
+  if (!pl || !workspace) return FP2_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  int32_t w[ST_WORDS];
+  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
+  if (cudaMemcpyAsync(w, ws + pl->ws_status, sizeof(w), cudaMemcpyDeviceToHost, st) != cudaSuccess) return FP2_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return FP2_ERR_CUDA;
+  if (cudaMemsetAsync(ws + pl->ws_status, 0, sizeof(w), st) != cudaSuccess) return FP2_ERR_CUDA;
+  if (h_words) memcpy(h_words, w, sizeof(w));
+  if (w[ST_TIMEOUT]) return FP2_ERR_TIMEOUT;
+  if (w[ST_BAD_LIST]) return FP2_ERR_INVALID_ARG;
+  return FP2_OK;
+}

@@ -1,0 +1,167 @@
+// Block-mean pooling (Eq. 5; Algorithm 1 line 2): kbar_J, vbar_J = mean over the real tokens of KV block J,
+// read through the page table (Eq. 22).  HBM-bound: K and V are read exactly once with 16-byte loads,
+// 256-byte (BF16) or 128-byte (FP8) contiguous per token row, fp32 accumulation.
+//
+// Outputs, all BF16 [nblk_tot, Hkv, 128]:
+//   kbar_hi = bf16(mean k), kbar_lo = bf16(mean k - kbar_hi)   (hi + lo carries ~16 mantissa bits for the scorer)
+//   vbar    = bf16(mean v)
+// kbar_hi and vbar double as the operands of the correction chunks in the attention kernel.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp8.h>
+#include "common.cuh"
+
+namespace fp2 {
+
+template <bool FP8>
+__device__ __forceinline__ void accum16(const uint4& v, float* acc) {
+  if constexpr (!FP8) {
+    const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&v);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float2 f = __bfloat1622float2(p[i]);
+      acc[2 * i] += f.x;
+      acc[2 * i + 1] += f.y;
+    }
+  } else {
+    const __nv_fp8x2_storage_t* p = reinterpret_cast<const __nv_fp8x2_storage_t*>(&v);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      __half2_raw h = __nv_cvt_fp8x2_to_halfraw2(p[i], __NV_E4M3);
+      float2 f = __half22float2(*reinterpret_cast<__half2*>(&h));
+      acc[2 * i] += f.x;
+      acc[2 * i + 1] += f.y;
+    }
+  }
+}
+
+// grid (nblk_tot, Hkv), 256 threads.
+template <bool FP8>
+__global__ void __launch_bounds__(256) pool_kv_kernel(const uint8_t* __restrict__ k_cache,
+                                                      const uint8_t* __restrict__ v_cache,
+                                                      const int32_t* __restrict__ page_table,
+                                                      const int32_t* __restrict__ seqlens_k,
+                                                      const int32_t* __restrict__ blk_off,  // [ns+1]
+                                                      const float* __restrict__ k_scale,
+                                                      const float* __restrict__ v_scale, DevParams P,
+                                                      __nv_bfloat16* __restrict__ kbar_hi,
+                                                      __nv_bfloat16* __restrict__ kbar_lo,
+                                                      __nv_bfloat16* __restrict__ vbar) {
+  constexpr int ROW_BYTES = FP8 ? 128 : 256;
+  constexpr int CHUNKS = ROW_BYTES / 16;       // 16-byte chunks per token row
+  constexpr int EPC = FP8 ? 16 : 8;            // elements per chunk
+  constexpr int ROWS_PER_PASS = 256 / CHUNKS;  // 16 (bf16) or 32 (fp8)
+  constexpr int PASSES = kBlock / ROWS_PER_PASS;
+
+  __shared__ float red[2][ROWS_PER_PASS][kHeadDim + 4];
+
+  const int gblk = blockIdx.x, h = blockIdx.y;
+  // sequence of this pooled block: binary search in blk_off
+  int lo = 0, hi = P.num_seqs;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (blk_off[mid] <= gblk) lo = mid; else hi = mid;
+  }
+  const int b = lo, J = gblk - blk_off[b];
+  const int Lk = seqlens_k[b];
+  const int ntok = min(kBlock, Lk - J * kBlock);
+  const int chunk = threadIdx.x % CHUNKS, rg = threadIdx.x / CHUNKS;
+  const int32_t* pt = page_table + (size_t)b * P.max_pages_per_seq;
+  const size_t row_stride = (size_t)P.num_kv_heads * ROW_BYTES;
+
+  float ak[EPC], av[EPC];
+#pragma unroll
+  for (int i = 0; i < EPC; ++i) ak[i] = av[i] = 0.f;
+
+  uint4 kv[PASSES], vv[PASSES];
+#pragma unroll
+  for (int ps = 0; ps < PASSES; ++ps) {
+    const int tl = ps * ROWS_PER_PASS + rg;
+    kv[ps] = make_uint4(0, 0, 0, 0);
+    vv[ps] = make_uint4(0, 0, 0, 0);
+    if (tl < ntok) {
+      const int j = J * kBlock + tl;
+      const size_t slot = (size_t)pt[j / P.page_size] * P.page_size + (j % P.page_size);
+      const size_t off = slot * row_stride + (size_t)h * ROW_BYTES + chunk * 16;
+      kv[ps] = __ldg(reinterpret_cast<const uint4*>(k_cache + off));
+      vv[ps] = __ldg(reinterpret_cast<const uint4*>(v_cache + off));
+    }
+  }
+#pragma unroll
+  for (int ps = 0; ps < PASSES; ++ps) {   // zero bit patterns add 0 in both encodings
+    accum16<FP8>(kv[ps], ak);
+    accum16<FP8>(vv[ps], av);
+  }
+#pragma unroll
+  for (int i = 0; i < EPC; ++i) {
+    red[0][rg][chunk * EPC + i] = ak[i];
+    red[1][rg][chunk * EPC + i] = av[i];
+  }
+  __syncthreads();
+  const int which = threadIdx.x / kHeadDim, c = threadIdx.x % kHeadDim;
+  float s = 0.f;
+#pragma unroll
+  for (int r = 0; r < ROWS_PER_PASS; ++r) s += red[which][r][c];
+  float mean = s / (float)ntok;
+  if constexpr (FP8) mean *= (which == 0 ? k_scale[h] : v_scale[h]);
+  const size_t o = ((size_t)gblk * P.num_kv_heads + h) * kHeadDim + c;
+  const __nv_bfloat16 hi16 = __float2bfloat16_rn(mean);
+  if (which == 0) {
+    kbar_hi[o] = hi16;
+    kbar_lo[o] = __float2bfloat16_rn(mean - __bfloat162float(hi16));
+  } else {
+    vbar[o] = hi16;
+  }
+}
+
+// ----------------------------------------------------------------------------------------
+// Work ordering (Sec. 3.3 "Sparsity-Aware Load Balancing", Eq. 21): segments sorted KV-head-major, then by
+// descending block count (capped), by a counting sort on the device.  Order among equal keys is arbitrary;
+// it only changes which CTA runs a segment, never a result.
+// ----------------------------------------------------------------------------------------
+__device__ __forceinline__ int order_bucket(int h, int count) {
+  int c = count < kCountBuckets - 1 ? count : kCountBuckets - 1;
+  return h * kCountBuckets + (kCountBuckets - 1 - c);
+}
+
+__global__ void order_hist_kernel(const SegInfo* __restrict__ segs, const int32_t* __restrict__ count, int nseg,
+                                  int32_t* __restrict__ hist) {
+  int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= nseg) return;
+  int c = count ? count[s] : segs[s].J_hi + 1;
+  atomicAdd(&hist[order_bucket(segs[s].h, c)], 1);
+}
+
+// single CTA of 1024 threads: exclusive scan of nb = Hkv * kCountBuckets counters, in place.
+__global__ void order_scan_kernel(int32_t* __restrict__ hist, int nb) {
+  __shared__ int32_t part[1024];
+  const int per = (nb + 1023) / 1024;
+  const int beg = threadIdx.x * per, end = min(beg + per, nb);
+  int s = 0;
+  for (int i = beg; i < end; ++i) s += hist[i];
+  part[threadIdx.x] = s;
+  __syncthreads();
+  for (int d = 1; d < 1024; d <<= 1) {
+    int v = threadIdx.x >= d ? part[threadIdx.x - d] : 0;
+    __syncthreads();
+    part[threadIdx.x] += v;
+    __syncthreads();
+  }
+  int run = part[threadIdx.x] - s;
+  for (int i = beg; i < end; ++i) {
+    int v = hist[i];
+    hist[i] = run;
+    run += v;
+  }
+}
+
+__global__ void order_scatter_kernel(const SegInfo* __restrict__ segs, const int32_t* __restrict__ count, int nseg,
+                                     int32_t* __restrict__ cursor, int32_t* __restrict__ order) {
+  int s = blockIdx.x * blockDim.x + threadIdx.x;
+  if (s >= nseg) return;
+  int c = count ? count[s] : segs[s].J_hi + 1;
+  int pos = atomicAdd(&cursor[order_bucket(segs[s].h, c)], 1);
+  order[pos] = s;
+}
+
+}  // namespace fp2

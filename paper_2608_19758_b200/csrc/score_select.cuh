@@ -1,0 +1,266 @@
+// Fused block scoring and selection (Eq. 19, Eq. 20; Algorithm 1 lines 3-5), one CTA per segment.
+//
+// For the packed query tile I (128 rows of one KV head) and every candidate block J <= J_hi:
+//     s_iJ = scale * q_i . kbar_J,   m_J = max_i s_iJ,   S_J = sum_i 2^{(s_iJ - m_J) log2 e}
+// (the per-block max / sum of Eq. 1), then  M = max_J m_J,  E_J = S_J 2^{(m_J - M) log2 e}  (the global
+// rescale of Eq. 2 / Eq. 20), threshold alpha * max_J E_J, forced sink / window / diagonal blocks, and an
+// ordered compaction of the survivors into the segment's list.
+//
+// The contraction runs on the tensor cores TRANSPOSED: A = a chunk of 128 pooled keys (rows = TMEM lanes),
+// B = the query tile (columns), so that each consumer thread owns one pooled key and the sum over the tile's
+// rows is a sum over its own TMEM columns -- no cross-thread reduction in the main loop.  kbar enters as a
+// BF16 (hi, lo) pair accumulated into the same fp32 accumulator, which keeps the energies accurate to ~1e-5
+// relative; a single BF16 kbar would move them by ~3e-3 and flip list entries.
+//
+// Roles: warps 0-3 / 4-7 = two consumer warpgroups alternating over chunks (TMEM accumulators 0 / 1),
+// warp 8 = TMA producer of kbar chunks, warp 9 = UMMA issuer.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp8.h>
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace fp2 {
+
+constexpr int kScoreThreads = 320;
+constexpr int kScoreStageBytes = 65536;  // kbar_hi chunk (32 KB) + kbar_lo chunk (32 KB)
+constexpr int kScoreSmemBytes = 1024 /*align*/ + 32768 /*Q*/ + 2 * kScoreStageBytes + 2 * kMaxBlocks * 4 + 1024;
+
+// Query tile -> shared memory in the K-major 128-byte-swizzled layout the UMMA descriptors expect:
+// BF16: two 64-column halves of [128 rows x 128 B]; FP8 is widened to BF16 on the way (exact).
+// Rows >= nrows are zero-filled.  Called by `nthr` threads with local index `t`.
+template <bool FP8, int BATCH = 8>
+__device__ __forceinline__ void load_q_tile_bf16(uint8_t* sQ, const uint8_t* __restrict__ q, const SegInfo& sg,
+                                                 const DevParams& P, int t, int nthr) {
+  const int g = P.group;
+  for (int i0 = t; i0 < kTileRows * 16; i0 += nthr * BATCH) {
+    uint4 v[BATCH];
+#pragma unroll
+    for (int u = 0; u < BATCH; ++u) {
+      const int i = i0 + u * nthr;
+      const int row = i >> 4, ch = i & 15;  // 16 chunks of 8 elements per row
+      v[u] = make_uint4(0, 0, 0, 0);
+      if (i < kTileRows * 16 && row < sg.nrows) {
+        const int r = sg.r0 + row;
+        const size_t tok = (size_t)sg.q_tok0 + r / g;
+        const size_t head = (size_t)sg.h * g + r % g;
+        const size_t e = (tok * P.num_q_heads + head) * kHeadDim + ch * 8;
+        if constexpr (!FP8) {
+          v[u] = __ldg(reinterpret_cast<const uint4*>(q + e * 2));
+        } else {
+          uint2 raw = __ldg(reinterpret_cast<const uint2*>(q + e));
+          const __nv_fp8x2_storage_t* p2 = reinterpret_cast<const __nv_fp8x2_storage_t*>(&raw);
+          uint32_t o[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            __half2_raw hh = __nv_cvt_fp8x2_to_halfraw2(p2[k], __NV_E4M3);
+            float2 f = __half22float2(*reinterpret_cast<__half2*>(&hh));
+            o[k] = pack_bf16x2(f.x, f.y);
+          }
+          v[u] = make_uint4(o[0], o[1], o[2], o[3]);
+        }
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < BATCH; ++u) {
+      const int i = i0 + u * nthr;
+      const int row = i >> 4, ch = i & 15;
+      if (i < kTileRows * 16)
+        *reinterpret_cast<uint4*>(sQ + (ch >> 3) * 16384 + sw128_offset(row, ch & 7)) = v[u];
+    }
+  }
+}
+
+template <bool FP8>
+__global__ void __launch_bounds__(kScoreThreads, 1)
+score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_constant__ CUtensorMap map_klo,
+                    const uint8_t* __restrict__ q, const SegInfo* __restrict__ segs, const float* __restrict__ q_scale,
+                    DevParams P, int64_t* __restrict__ seg_offset, int32_t* __restrict__ seg_count,
+                    int32_t* __restrict__ blk_idx, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem;
+  uint8_t* sStage = smem + 32768;
+  float* sS = reinterpret_cast<float*>(sStage + 2 * kScoreStageBytes);  // per candidate: S_J, later E_J
+  float* sM = sS + kMaxBlocks;                                          // per candidate: m_J
+  float* sC = sM + kMaxBlocks;                                          // per tile row: logit multiplier (FP8)
+
+  __shared__ uint64_t full[2], empty[2], acc_full[2], acc_empty[2];
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_flag;
+  __shared__ float red[8];
+  __shared__ int wsum[8];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // heaviest tiles (largest candidate count) of every sequence come last in segment order: launch them first
+  const int seg = P.nseg - 1 - (int)blockIdx.x;
+  const SegInfo sg = segs[seg];
+  const int ncand = sg.J_hi + 1;
+  const int nchunks = (ncand + 127) >> 7;
+  WaitCtx ctx{status, &abort_flag};
+
+  if (tid == 0) {
+    abort_flag = 0;
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], 1);
+      mbar_init(&acc_full[i], 1);
+      mbar_init(&acc_empty[i], 128);
+    }
+    fence_barrier_init();
+  }
+  if (warp == 9) {
+    tmem_alloc(&tmem_base_s, 256);
+    tmem_relinquish();
+  }
+  if (warp < 8) {
+    load_q_tile_bf16<FP8>(sQ, q, sg, P, tid, 256);
+    if constexpr (FP8) {
+      if (tid < kTileRows) {
+        const int r = sg.r0 + tid;
+        sC[tid] = P.scale_log2 * q_scale[sg.h * P.group + r % P.group];
+      }
+    }
+    fence_proxy_async();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base_s;
+
+  if (warp == 8) {
+    // ---------------- producer: kbar chunks (hi and lo) via TMA ----------------
+    if (lane == 0) {
+      tma_prefetch_desc(&map_khi);
+      tma_prefetch_desc(&map_klo);
+      for (int c = 0; c < nchunks; ++c) {
+        const int s = c & 1;
+        if (c >= 2) mbar_wait(&empty[s], ((c >> 1) - 1) & 1, ctx, 101);
+        uint8_t* dst = sStage + s * kScoreStageBytes;
+        mbar_arrive_expect_tx(&full[s], kScoreStageBytes);
+        const int row0 = sg.blk_off + c * 128;
+        tma_load_3d(dst, &map_khi, &full[s], 0, sg.h, row0);
+        tma_load_3d(dst + 16384, &map_khi, &full[s], 64, sg.h, row0);
+        tma_load_3d(dst + 32768, &map_klo, &full[s], 0, sg.h, row0);
+        tma_load_3d(dst + 49152, &map_klo, &full[s], 64, sg.h, row0);
+      }
+    }
+  } else if (warp == 9) {
+    // ---------------- UMMA issuer: acc[c&1] = kbar_hi Q^T + kbar_lo Q^T ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(128, 128, 1, 1, 0, 0);
+      const uint32_t q_addr = smem_u32(sQ);
+      for (int c = 0; c < nchunks; ++c) {
+        const int s = c & 1;
+        mbar_wait(&full[s], (c >> 1) & 1, ctx, 102);
+        if (c >= 2) mbar_wait(&acc_empty[s], ((c >> 1) - 1) & 1, ctx, 103);
+        tc_fence_after();
+        const uint32_t a_addr = smem_u32(sStage + s * kScoreStageBytes);
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+            const uint64_t ad = make_smem_desc_sw128(a_addr + part * 32768 + off, 16, 1024);
+            const uint64_t bd = make_smem_desc_sw128(q_addr + off, 16, 1024);
+            umma_f16_ss(tmem + s * 128, ad, bd, idesc, (part | ks) != 0);
+          }
+        }
+        umma_commit(&empty[s]);
+        umma_commit(&acc_full[s]);
+      }
+    }
+  } else {
+    // ---------------- consumers: per pooled key, max and exp-sum over the tile's rows ----------------
+    const int wg = warp >> 2;
+    const int key = (warp & 3) * 32 + lane;  // TMEM lane = pooled key within the chunk
+    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + wg * 128;
+    const float cs = P.scale_log2;
+    for (int c = wg; c < nchunks; c += 2) {
+      mbar_wait(&acc_full[wg], (c >> 1) & 1, ctx, 104);
+      tc_fence_after();
+      float x[128];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        uint32_t r[32];
+        tmem_ld32(lane_addr + k * 32, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) x[k * 32 + j] = __uint_as_float(r[j]);
+      }
+      tc_fence_before();
+      mbar_arrive(&acc_empty[wg]);
+      float m = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 128; ++j) {
+        float mult = cs;
+        if constexpr (FP8) mult = sC[j];
+        x[j] = (j < sg.nrows) ? x[j] * mult : -INFINITY;
+        m = fmaxf(m, x[j]);
+      }
+      float sum = 0.f;
+#pragma unroll
+      for (int j = 0; j < 128; ++j) sum += ex2(x[j] - m);
+      const int J = c * 128 + key;
+      if (J < ncand) {
+        sS[J] = sum;
+        sM[J] = m;
+      }
+    }
+    // ---------------- selection: all 256 consumer threads ----------------
+    named_bar_sync(1, 256);
+    float lm = -INFINITY;
+    for (int J = tid; J < ncand; J += 256) lm = fmaxf(lm, sM[J]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) lm = fmaxf(lm, __shfl_xor_sync(0xffffffffu, lm, o));
+    if (lane == 0) red[warp] = lm;
+    named_bar_sync(1, 256);
+    float M = red[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) M = fmaxf(M, red[i]);
+    named_bar_sync(1, 256);
+    float le = 0.f;
+    for (int J = tid; J < ncand; J += 256) {
+      const float e = sS[J] * exp2f(sM[J] - M);
+      sS[J] = e;
+      le = fmaxf(le, e);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) le = fmaxf(le, __shfl_xor_sync(0xffffffffu, le, o));
+    if (lane == 0) red[warp] = le;
+    named_bar_sync(1, 256);
+    float maxE = red[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) maxE = fmaxf(maxE, red[i]);
+    const float thr = P.alpha * maxE;
+    const int win_lo = sg.J_lo - P.window_blocks;
+    int base = 0;
+    for (int J0 = 0; J0 < ncand; J0 += 256) {
+      const int J = J0 + tid;
+      const bool keep = J < ncand && (sS[J] >= thr || J < P.sink_blocks || J >= win_lo);
+      const unsigned bal = __ballot_sync(0xffffffffu, keep);
+      if (lane == 0) wsum[warp] = __popc(bal);
+      named_bar_sync(1, 256);
+      int before = 0, total = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int v = wsum[i];
+        before += (i < warp) ? v : 0;
+        total += v;
+      }
+      if (keep) blk_idx[sg.off + base + before + __popc(bal & ((1u << lane) - 1u))] = J;
+      base += total;
+      named_bar_sync(1, 256);
+    }
+    if (tid == 0) {
+      seg_count[seg] = base;
+      seg_offset[seg] = sg.off;
+      if (seg == P.nseg - 1) seg_offset[P.nseg] = sg.off + ncand;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) tmem_dealloc(tmem, 256);
+}
+
+}  // namespace fp2
