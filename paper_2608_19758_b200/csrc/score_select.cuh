@@ -71,6 +71,39 @@ __device__ __forceinline__ void load_q_tile_bf16(uint8_t* sQ, const uint8_t* __r
   }
 }
 
+// One pooled key (= this thread's TMEM lane) against the 128 query rows of the tile (= TMEM columns):
+// m = max_j x_j, sum = sum_j 2^(x_j - m), x_j = s_j * (scale log2 e [* q_scale of row j]).  PARTIAL: only the
+// first nrows columns are real query rows.  Releases the accumulator as soon as it is in registers.
+template <bool FP8, bool PARTIAL>
+__device__ __forceinline__ void score_chunk(uint32_t lane_addr, float cs, const float* sC, int nrows,
+                                            uint64_t* acc_empty_bar, float& m_out, float& sum_out) {
+  uint32_t xv[128];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) tmem_ld32(lane_addr + k * 32, reinterpret_cast<uint32_t(&)[32]>(xv[k * 32]));
+  tmem_wait_ld();
+  tc_fence_before();
+  mbar_arrive(acc_empty_bar);
+  float x[128];
+#pragma unroll
+  for (int j = 0; j < 128; ++j) {
+    float mult = cs;
+    if constexpr (FP8) mult = sC[j];
+    x[j] = __uint_as_float(xv[j]) * mult;
+    if constexpr (PARTIAL) x[j] = (j < nrows) ? x[j] : -INFINITY;
+  }
+  float m8[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) m8[j] = x[j];
+#pragma unroll
+  for (int j = 8; j < 128; ++j) m8[j & 7] = fmaxf(m8[j & 7], x[j]);
+  const float m = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
+  float s8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+  for (int j = 0; j < 128; ++j) s8[j & 7] += ex2(x[j] - m);
+  m_out = m;
+  sum_out = ((s8[0] + s8[1]) + (s8[2] + s8[3])) + ((s8[4] + s8[5]) + (s8[6] + s8[7]));
+}
+
 template <bool FP8>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_constant__ CUtensorMap map_klo,
@@ -179,28 +212,9 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
     for (int c = wg; c < nchunks; c += 2) {
       mbar_wait(&acc_full[wg], (c >> 1) & 1, ctx, 104);
       tc_fence_after();
-      float x[128];
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        uint32_t r[32];
-        tmem_ld32(lane_addr + k * 32, r);
-        tmem_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) x[k * 32 + j] = __uint_as_float(r[j]);
-      }
-      tc_fence_before();
-      mbar_arrive(&acc_empty[wg]);
-      float m = -INFINITY;
-#pragma unroll
-      for (int j = 0; j < 128; ++j) {
-        float mult = cs;
-        if constexpr (FP8) mult = sC[j];
-        x[j] = (j < sg.nrows) ? x[j] * mult : -INFINITY;
-        m = fmaxf(m, x[j]);
-      }
-      float sum = 0.f;
-#pragma unroll
-      for (int j = 0; j < 128; ++j) sum += ex2(x[j] - m);
+      float m, sum;
+      if (sg.nrows == kTileRows) score_chunk<FP8, false>(lane_addr, cs, sC, kTileRows, &acc_empty[wg], m, sum);
+      else score_chunk<FP8, true>(lane_addr, cs, sC, sg.nrows, &acc_empty[wg], m, sum);
       const int J = c * 128 + key;
       if (J < ncand) {
         sS[J] = sum;

@@ -59,6 +59,94 @@ struct AttnArgs {
   int* status;
 };
 
+// Masked iterations (diagonal blocks, correction chunks -- the minority): overwrite the hidden logits of this
+// thread's row with -inf in TMEM, so that the softmax step itself carries no mask logic.  Column j stays
+// visible iff j <= tok_lim and bit j of cm is set.  (Predicating the mask into the softmax body cost 2.5x on
+// every iteration, masked or not.)
+__device__ __forceinline__ void mask_tile(uint32_t s_addr, int tok_lim, const uint32_t* cm) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const bool all_vis = (k * 32 + 31 <= tok_lim) && (cm[k] == 0xffffffffu);
+    if (__all_sync(0xffffffffu, all_vis)) continue;
+    uint32_t rr[32];
+    tmem_ld32(s_addr + k * 32, rr);
+    tmem_wait_ld();
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const bool vis = (k * 32 + j <= tok_lim) && ((cm[k] >> j) & 1u);
+      rr[j] = vis ? rr[j] : 0xff800000u;  // -inf
+    }
+    tmem_st32(s_addr + k * 32, rr);
+  }
+  tmem_wait_st();
+}
+
+// Online-softmax step of one thread (= one query row) over a 128-column logit tile held in TMEM at s_addr:
+// updates the running maximum m (log2 units) and sum l, rescales the row of the O accumulator at o_addr when
+// the maximum moved by more than 2^8 (lazy rescale; decided per warp because TMEM accesses are warp-wide),
+// and overwrites the first 64 columns of the tile with P = 2^(x - m) as BF16 pairs (the A operand of P V).
+//   x_j = s_j * cs + shift
+__device__ __forceinline__ void softmax_tile(uint32_t s_addr, uint32_t o_addr, float cs, float shift, bool have_o,
+                                             float& m, float& l) {
+  // pass 1: row maximum.  Four TMEM loads in flight behind one wait, eight independent max chains.
+  float mx;
+  {
+    uint32_t sv[128];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) tmem_ld32(s_addr + k * 32, reinterpret_cast<uint32_t(&)[32]>(sv[k * 32]));
+    tmem_wait_ld();
+    float mx8[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) mx8[c] = __uint_as_float(sv[c]);
+#pragma unroll
+    for (int j = 8; j < 128; ++j) mx8[j & 7] = fmaxf(mx8[j & 7], __uint_as_float(sv[j]));
+    mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
+               fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+  }
+  mx = fmaf(mx, cs, shift);  // cs > 0: scaling commutes with the maximum
+  const float m_new = fmaxf(m, mx);
+  const bool need = m_new > m + 8.0f;
+  if (__any_sync(0xffffffffu, need)) {
+    const float f = (m == -INFINITY) ? 0.f : ex2(m - m_new);
+    if (have_o) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        uint32_t rr[32];
+        tmem_ld32(o_addr + k * 32, rr);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; ++j) rr[j] = __float_as_uint(__uint_as_float(rr[j]) * f);
+        tmem_st32(o_addr + k * 32, rr);
+      }
+    }
+    l *= f;
+    m = m_new;
+  }
+  // pass 2: p = 2^(x - m).  Chunk k of P lands on columns [16k, 16k+16), which pass 2 has already read; the
+  // load of chunk k+1 is in flight while chunk k is exponentiated.  A row with nothing visible so far has
+  // m = -inf and only -inf logits: its exponent is taken against 0 and gives exact zeros.
+  const float neg_m = (m == -INFINITY) ? shift : shift - m;
+  float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+  uint32_t buf[2][32];
+  tmem_ld32(s_addr, buf[0]);
+  tmem_wait_ld();
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    if (k < 3) tmem_ld32(s_addr + (k + 1) * 32, buf[(k + 1) & 1]);
+    uint32_t pk[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const float p0 = ex2(fmaf(__uint_as_float(buf[k & 1][2 * j]), cs, neg_m));
+      const float p1 = ex2(fmaf(__uint_as_float(buf[k & 1][2 * j + 1]), cs, neg_m));
+      sum4[j & 3] += p0 + p1;
+      pk[j] = pack_bf16x2(p0, p1);
+    }
+    if (k < 3) tmem_wait_ld();
+    tmem_st16(s_addr + k * 16, pk);
+  }
+  l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+}
+
 template <bool FP8>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -341,6 +429,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       const int pos = sg.pre + r / g;
       float m = -INFINITY, l = 0.f;
       int used = 0;
+      // block id of this warpgroup's next exact iteration, fetched one iteration ahead
+      int J_next = (!ti.dense && wg < T) ? list[T - 1 - wg] : 0;
       for (int i = wg; i < n_it; i += 2, ++used) {
         // iteration kind and masks
         bool need_mask = false;
@@ -348,7 +438,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         uint32_t cm[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
         float shift = 0.f;
         if (i < T) {
-          int J = ti.dense ? sg.J_hi - i : list[T - 1 - i];
+          int J = ti.dense ? sg.J_hi - i : J_next;
+          if (!ti.dense && i + 2 < T) J_next = list[T - 3 - i];
           J = max(0, min(J, sg.J_hi));
           need_mask = J >= sg.J_lo;
           tok_lim = pos - J * kBlock;
@@ -363,70 +454,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         mbar_wait(&s_full[wg], sc & 1, ctx, 502);
         ++sc;
         tc_fence_after();
-        // pass 1: row maximum of the masked, scaled logits (32 columns at a time)
-        float mx = -INFINITY;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          uint32_t rr[32];
-          tmem_ld32(s_addr + k * 32, rr);
-          tmem_wait_ld();
-          if (need_mask) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const bool vis = (k * 32 + j <= tok_lim) && ((cm[k] >> j) & 1u);
-              mx = vis ? fmaxf(mx, __uint_as_float(rr[j])) : mx;
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(rr[j]));
-          }
-        }
-        mx = fmaf(mx, cs, shift);  // cs > 0: scaling commutes with the maximum
-        const float m_new = fmaxf(m, mx);
-        // lazy rescale: only when some row of the warp moved its maximum by more than 2^8
-        const bool need = m_new > m + 8.0f;
-        if (__any_sync(0xffffffffu, need)) {
-          const float f = (m == -INFINITY) ? 0.f : ex2(m - m_new);
-          if (used > 0) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              uint32_t rr[32];
-              tmem_ld32(o_addr + k * 32, rr);
-              tmem_wait_ld();
-#pragma unroll
-              for (int j = 0; j < 32; ++j) rr[j] = __float_as_uint(__uint_as_float(rr[j]) * f);
-              tmem_st32(o_addr + k * 32, rr);
-            }
-          }
-          l *= f;
-          m = m_new;
-        }
-        // pass 2: p = 2^(x - m), written back as BF16 pairs over the first 64 columns of S (chunk k of P
-        // lands on columns [16k, 16k+16), all of which pass 2 has already read)
-        const float neg_m = (m == -INFINITY) ? shift : shift - m;
-        float sum = 0.f;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          uint32_t rr[32];
-          tmem_ld32(s_addr + k * 32, rr);
-          tmem_wait_ld();
-          uint32_t pk[16];
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            float p0 = ex2(fmaf(__uint_as_float(rr[2 * j]), cs, neg_m));
-            float p1 = ex2(fmaf(__uint_as_float(rr[2 * j + 1]), cs, neg_m));
-            if (need_mask) {
-              const bool v0 = (k * 32 + 2 * j <= tok_lim) && ((cm[k] >> (2 * j)) & 1u);
-              const bool v1 = (k * 32 + 2 * j + 1 <= tok_lim) && ((cm[k] >> (2 * j + 1)) & 1u);
-              p0 = v0 ? p0 : 0.f;
-              p1 = v1 ? p1 : 0.f;
-            }
-            sum += p0 + p1;
-            pk[j] = pack_bf16x2(p0, p1);
-          }
-          tmem_st16(s_addr + k * 16, pk);
-        }
-        l += sum;
+        if (need_mask) mask_tile(s_addr, tok_lim, cm);
+        softmax_tile(s_addr, o_addr, cs, shift, used > 0, m, l);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&p_ready[wg]);
