@@ -9,16 +9,19 @@
 // shifted by log2(128) (every corrected block is full) and masked by todo = fully-visible & ~selected.
 //
 // Roles (12 warps):
-//   warps 0-3  softmax warpgroup 0: iterations 0, 2, 4, ...  (TMEM: S0 / P0, O0)
-//   warps 4-7  softmax warpgroup 1: iterations 1, 3, 5, ...  (TMEM: S1 / P1, O1)
-//       each keeps its own running (max, sum) and its own O accumulator; the two are merged in the epilogue,
-//       so the warpgroups never synchronise inside the main loop and one's exponentials overlap the other's MMAs.
+//   warps 0-7  two softmax warpgroups.  Both work on EVERY iteration: warpgroup w owns logit columns
+//              [64w, 64w+64) of all 128 rows (thread = row).  They exchange the row maximum through shared
+//              memory once per iteration, so the softmax latency of a block is halved and one accumulator O
+//              serves the whole tile (no merge at the end).
 //   warp 8     TMA producer: K / V pages through the page table into two rings (Eq. 22)
 //   warp 9     UMMA issuer: S = Q K^T (SS), O += P V (P read from TMEM, V MN-major from shared memory)
 //   warps 10-11 tile set-up: fetch the next unit, validate its list, build the correction masks, stage Q
 //
-// TMEM columns: S0 [0,128) S1 [128,256) O0 [256,384) O1 [384,512); P (BF16 pairs) overwrites the first 64
-// columns of its S buffer.
+// TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512).  P (BF16 pairs) has its own
+// columns, so S = Q K^T of iteration i+2 may start as soon as the softmax of iteration i has read S -- it does
+// not wait for O += P V of iteration i.  Issue order: QK(0) QK(1) PV(0) QK(2) PV(1) ...  Measured on B200:
+// consecutive UMMAs that differ in instruction descriptor or A source drain the pipe (~245 cycles), which
+// bounds this order at ~1510 cycles per 128x128 block against 1024 for back-to-back MMAs.
 #pragma once
 #include <cuda_bf16.h>
 #include "common.cuh"
@@ -31,7 +34,7 @@ constexpr int kAttnThreads = 384;
 constexpr int kNK = 3;  // K ring stages (32 KB each)
 constexpr int kNV = 2;  // V ring stages
 constexpr int kTileBytes = 32768;
-constexpr int kAttnSmemBytes = 1024 + kTileBytes * (1 + kNK + kNV) + 2048;
+constexpr int kAttnSmemBytes = 1024 + kTileBytes * (1 + kNK + kNV) + 3072;
 
 struct TileInfo {
   SegInfo sg;
@@ -60,20 +63,21 @@ struct AttnArgs {
 };
 
 // Masked iterations (diagonal blocks, correction chunks -- the minority): overwrite the hidden logits of this
-// thread's row with -inf in TMEM, so that the softmax step itself carries no mask logic.  Column j stays
-// visible iff j <= tok_lim and bit j of cm is set.  (Predicating the mask into the softmax body cost 2.5x on
-// every iteration, masked or not.)
-__device__ __forceinline__ void mask_tile(uint32_t s_addr, int tok_lim, const uint32_t* cm) {
+// thread's row with -inf in TMEM, so that the softmax step itself carries no mask logic (predicating the mask
+// into the softmax body cost 2.5x on every iteration, masked or not).  The thread owns 64 columns starting at
+// block column col0; column j stays visible iff j <= tok_lim and bit (j - col0) of {cm_lo, cm_hi} is set.
+__device__ __forceinline__ void mask_half(uint32_t s_addr, int col0, int tok_lim, uint32_t cm_lo, uint32_t cm_hi) {
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    const bool all_vis = (k * 32 + 31 <= tok_lim) && (cm[k] == 0xffffffffu);
-    if (__all_sync(0xffffffffu, all_vis)) continue;
+  for (int k = 0; k < 2; ++k) {
+    const uint32_t cm = k ? cm_hi : cm_lo;
+    const bool all_vis = (col0 + k * 32 + 31 <= tok_lim) && (cm == 0xffffffffu);
+    if (__all_sync(0xffffffffu, all_vis)) continue;   // TMEM accesses are warp-wide: decide per warp
     uint32_t rr[32];
     tmem_ld32(s_addr + k * 32, rr);
     tmem_wait_ld();
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
-      const bool vis = (k * 32 + j <= tok_lim) && ((cm[k] >> j) & 1u);
+      const bool vis = (col0 + k * 32 + j <= tok_lim) && ((cm >> j) & 1u);
       rr[j] = vis ? rr[j] : 0xff800000u;  // -inf
     }
     tmem_st32(s_addr + k * 32, rr);
@@ -81,70 +85,42 @@ __device__ __forceinline__ void mask_tile(uint32_t s_addr, int tok_lim, const ui
   tmem_wait_st();
 }
 
-// Online-softmax step of one thread (= one query row) over a 128-column logit tile held in TMEM at s_addr:
-// updates the running maximum m (log2 units) and sum l, rescales the row of the O accumulator at o_addr when
-// the maximum moved by more than 2^8 (lazy rescale; decided per warp because TMEM accesses are warp-wide),
-// and overwrites the first 64 columns of the tile with P = 2^(x - m) as BF16 pairs (the A operand of P V).
-//   x_j = s_j * cs + shift
-__device__ __forceinline__ void softmax_tile(uint32_t s_addr, uint32_t o_addr, float cs, float shift, bool have_o,
-                                             float& m, float& l) {
-  // pass 1: row maximum.  Four TMEM loads in flight behind one wait, eight independent max chains.
-  float mx;
-  {
-    uint32_t sv[128];
+// Row maximum of this thread's 64 logit columns (raw, unscaled): two TMEM loads in flight, eight max chains.
+__device__ __forceinline__ float half_row_max(uint32_t s_addr) {
+  uint32_t sv[64];
+  tmem_ld32(s_addr, reinterpret_cast<uint32_t(&)[32]>(sv[0]));
+  tmem_ld32(s_addr + 32, reinterpret_cast<uint32_t(&)[32]>(sv[32]));
+  tmem_wait_ld();
+  float mx8[8];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) tmem_ld32(s_addr + k * 32, reinterpret_cast<uint32_t(&)[32]>(sv[k * 32]));
-    tmem_wait_ld();
-    float mx8[8];
+  for (int c = 0; c < 8; ++c) mx8[c] = __uint_as_float(sv[c]);
 #pragma unroll
-    for (int c = 0; c < 8; ++c) mx8[c] = __uint_as_float(sv[c]);
-#pragma unroll
-    for (int j = 8; j < 128; ++j) mx8[j & 7] = fmaxf(mx8[j & 7], __uint_as_float(sv[j]));
-    mx = fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])),
-               fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
-  }
-  mx = fmaf(mx, cs, shift);  // cs > 0: scaling commutes with the maximum
-  const float m_new = fmaxf(m, mx);
-  const bool need = m_new > m + 8.0f;
-  if (__any_sync(0xffffffffu, need)) {
-    const float f = (m == -INFINITY) ? 0.f : ex2(m - m_new);
-    if (have_o) {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        uint32_t rr[32];
-        tmem_ld32(o_addr + k * 32, rr);
-        tmem_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 32; ++j) rr[j] = __float_as_uint(__uint_as_float(rr[j]) * f);
-        tmem_st32(o_addr + k * 32, rr);
-      }
-    }
-    l *= f;
-    m = m_new;
-  }
-  // pass 2: p = 2^(x - m).  Chunk k of P lands on columns [16k, 16k+16), which pass 2 has already read; the
-  // load of chunk k+1 is in flight while chunk k is exponentiated.  A row with nothing visible so far has
-  // m = -inf and only -inf logits: its exponent is taken against 0 and gives exact zeros.
-  const float neg_m = (m == -INFINITY) ? shift : shift - m;
+  for (int j = 8; j < 64; ++j) mx8[j & 7] = fmaxf(mx8[j & 7], __uint_as_float(sv[j]));
+  return fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])), fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+}
+
+// p = 2^(s * cs + neg_m) for this thread's 64 columns, written as BF16 pairs to 32 columns at p_addr.
+// The second TMEM load is in flight while the first half is exponentiated.  Returns the row's partial sum.
+__device__ __forceinline__ float half_row_exp(uint32_t s_addr, uint32_t p_addr, float cs, float neg_m) {
   float sum4[4] = {0.f, 0.f, 0.f, 0.f};
   uint32_t buf[2][32];
   tmem_ld32(s_addr, buf[0]);
   tmem_wait_ld();
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    if (k < 3) tmem_ld32(s_addr + (k + 1) * 32, buf[(k + 1) & 1]);
+  for (int k = 0; k < 2; ++k) {
+    if (k == 0) tmem_ld32(s_addr + 32, buf[1]);
     uint32_t pk[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      const float p0 = ex2(fmaf(__uint_as_float(buf[k & 1][2 * j]), cs, neg_m));
-      const float p1 = ex2(fmaf(__uint_as_float(buf[k & 1][2 * j + 1]), cs, neg_m));
+      const float p0 = ex2(fmaf(__uint_as_float(buf[k][2 * j]), cs, neg_m));
+      const float p1 = ex2(fmaf(__uint_as_float(buf[k][2 * j + 1]), cs, neg_m));
       sum4[j & 3] += p0 + p1;
       pk[j] = pack_bf16x2(p0, p1);
     }
-    if (k < 3) tmem_wait_ld();
-    tmem_st16(s_addr + k * 16, pk);
+    if (k == 0) tmem_wait_ld();
+    tmem_st16(p_addr + k * 16, pk);
   }
-  l += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+  return (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
 }
 
 template <bool FP8>
@@ -158,13 +134,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
   uint8_t* sQ = smem;
   uint8_t* sK = smem + kTileBytes;
   uint8_t* sV = sK + kNK * kTileBytes;
-  float* sML = reinterpret_cast<float*>(sV + kNV * kTileBytes);  // [2 wg][2 (m,l)][128]
+  float* sX = reinterpret_cast<float*>(sV + kNV * kTileBytes);   // [2 parity][2 wg][128] row-max / row-sum exchange
 
   __shared__ TileInfo info[2];
   __shared__ uint32_t sel_bits[2][kMaxBlocks / 32];
   __shared__ uint64_t info_full[2], info_empty[2], q_full, q_empty, tile_done;
   __shared__ uint64_t k_full[kNK], k_empty[kNK], v_full[kNV], v_empty[kNV];
-  __shared__ uint64_t s_full[2], p_ready[2];
+  __shared__ uint64_t s_full[2], p_ready[2], o_done;
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
 
@@ -177,11 +153,12 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       mbar_init(&info_full[i], 1);
       mbar_init(&info_empty[i], 2 + 256);
       mbar_init(&s_full[i], 1);
-      mbar_init(&p_ready[i], 128);
+      mbar_init(&p_ready[i], 256);
     }
     mbar_init(&q_full, 64);
     mbar_init(&q_empty, 1);
     mbar_init(&tile_done, 1);
+    mbar_init(&o_done, 1);
     for (int i = 0; i < kNK; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
     for (int i = 0; i < kNV; ++i) { mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); }
     fence_barrier_init();
@@ -358,11 +335,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       constexpr uint32_t idesc_qk = make_idesc(128, 128, 1, 1, 0, 0);
       constexpr uint32_t idesc_pv = make_idesc(128, 128, 1, 1, 0, 1);
       const uint32_t q_addr = smem_u32(sQ);
-      uint32_t kc = 0, vc = 0, pc[2] = {0, 0};
+      uint32_t kc = 0, vc = 0, pc0 = 0, pc1 = 0;
       auto issue_pv = [&](int j) {
         const int b = j & 1;
-        mbar_wait(&p_ready[b], pc[b] & 1, ctx, 401);
-        ++pc[b];
+        if (b) { mbar_wait(&p_ready[1], pc1 & 1, ctx, 401); ++pc1; }
+        else { mbar_wait(&p_ready[0], pc0 & 1, ctx, 401); ++pc0; }
         const int vs = vc % kNV;
         mbar_wait(&v_full[vs], (vc / kNV) & 1, ctx, 402);
         tc_fence_after();
@@ -370,9 +347,10 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
           const uint64_t bd = make_smem_desc_sw128(v_addr + ks * 2048, 16384, 1024);
-          umma_f16_ts(tmem + 256 + b * 128, tmem + b * 128 + ks * 8, bd, idesc_pv, (j >= 2) || ks > 0);
+          umma_f16_ts(tmem + 256, tmem + 384 + b * 64 + ks * 8, bd, idesc_pv, (j > 0) || ks > 0);
         }
         umma_commit(&v_empty[vs]);
+        umma_commit(&o_done);
         ++vc;
       };
       for (int it = 0;; ++it) {
@@ -388,6 +366,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           mbar_wait(&k_full[ks_], (kc / kNK) & 1, ctx, 405);
           tc_fence_after();
           const uint32_t k_addr = smem_u32(sK + ks_ * kTileBytes);
+          // S_a is free: the softmax of iteration i-2 signalled p_ready[a] (waited for in issue_pv(i-2))
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
             const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
@@ -413,9 +392,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     const int wg = warp >> 2;
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    const uint32_t s_addr = lane_base + wg * 128;
-    const uint32_t o_addr = lane_base + 256 + wg * 128;
-    uint32_t sc = 0;  // uses of this warpgroup's S buffer so far (phase of s_full[wg])
+    const uint32_t o_addr = lane_base + 256 + wg * 64;   // this thread's 64 columns of O
+    uint32_t sc0 = 0, sc1 = 0;   // completed uses of S0 / S1 (phases of s_full)
+    uint32_t pv_base = 0;        // UMMA groups O += P V issued before this tile (phase of o_done)
     const float cs = P.scale_log2;
     for (int it = 0;; ++it) {
       const int slot = it & 1;
@@ -428,75 +407,98 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       const int r = sg.r0 + row;
       const int pos = sg.pre + r / g;
       float m = -INFINITY, l = 0.f;
-      int used = 0;
-      // block id of this warpgroup's next exact iteration, fetched one iteration ahead
-      int J_next = (!ti.dense && wg < T) ? list[T - 1 - wg] : 0;
-      for (int i = wg; i < n_it; i += 2, ++used) {
+      // block id of the next exact iteration, fetched one iteration ahead
+      int J_next = (!ti.dense && T > 0) ? list[T - 1] : 0;
+      for (int i = 0; i < n_it; ++i) {
+        const int a = i & 1;
+        const uint32_t s_addr = lane_base + a * 128 + wg * 64;
+        const uint32_t p_addr = lane_base + 384 + a * 64 + wg * 32;
         // iteration kind and masks
         bool need_mask = false;
-        int tok_lim = 0;           // exact block: columns j with j <= tok_lim are visible
-        uint32_t cm[4] = {0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu};
+        int tok_lim = 1 << 30;     // exact block: columns j with j <= tok_lim are visible
+        uint32_t cm_lo = 0xffffffffu, cm_hi = 0xffffffffu;
         float shift = 0.f;
         if (i < T) {
           int J = ti.dense ? sg.J_hi - i : J_next;
-          if (!ti.dense && i + 2 < T) J_next = list[T - 3 - i];
+          if (!ti.dense && i + 1 < T) J_next = list[T - 2 - i];
           J = max(0, min(J, sg.J_hi));
           need_mask = J >= sg.J_lo;
           tok_lim = pos - J * kBlock;
         } else {
           const int c = ti.chunk_id[i - T];
-#pragma unroll
-          for (int w = 0; w < 4; ++w) cm[w] = ti.todo[c][w];
+          cm_lo = ti.todo[c][2 * wg];
+          cm_hi = ti.todo[c][2 * wg + 1];
           shift = 7.0f;  // log2(128): one pooled row stands for a full block (Eq. 6)
           need_mask = true;
-          tok_lim = 1 << 30;
         }
-        mbar_wait(&s_full[wg], sc & 1, ctx, 502);
-        ++sc;
+        if (a) { mbar_wait(&s_full[1], sc1 & 1, ctx, 502); ++sc1; }
+        else { mbar_wait(&s_full[0], sc0 & 1, ctx, 502); ++sc0; }
         tc_fence_after();
-        if (need_mask) mask_tile(s_addr, tok_lim, cm);
-        softmax_tile(s_addr, o_addr, cs, shift, used > 0, m, l);
+        if (need_mask) mask_half(s_addr, wg * 64, tok_lim, cm_lo, cm_hi);
+        // row maximum over all 128 columns: own half, then the other warpgroup's through shared memory
+        float mx = half_row_max(s_addr);
+        float* xch = sX + (i & 1) * 256;
+        xch[wg * 128 + row] = mx;
+        named_bar_sync(1, 256);
+        mx = fmaxf(mx, xch[(wg ^ 1) * 128 + row]);
+        mx = fmaf(mx, cs, shift);  // cs > 0: scaling commutes with the maximum
+        const float m_new = fmaxf(m, mx);
+        // lazy rescale: only when some row of the warp moved its maximum by more than 2^8.  Both warpgroups
+        // hold the same rows in the same warps and the same m, so they take the same decision.
+        const bool need = m_new > m + 8.0f;
+        if (__any_sync(0xffffffffu, need)) {
+          const float f = (m == -INFINITY) ? 0.f : ex2(m - m_new);
+          if (i > 0) {
+            // O must be at rest: wait for O += P V of iteration i-1 (UMMA group number pv_base + i)
+            mbar_wait(&o_done, (pv_base + i - 1) & 1, ctx, 504);
+            tc_fence_after();
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+              uint32_t rr[32];
+              tmem_ld32(o_addr + k * 32, rr);
+              tmem_wait_ld();
+#pragma unroll
+              for (int j = 0; j < 32; ++j) rr[j] = __float_as_uint(__uint_as_float(rr[j]) * f);
+              tmem_st32(o_addr + k * 32, rr);
+            }
+          }
+          l *= f;
+          m = m_new;
+        }
+        // a row with nothing visible so far has m = -inf and only -inf logits: exponent against 0 -> zeros
+        const float neg_m = (m == -INFINITY) ? shift : shift - m;
+        l += half_row_exp(s_addr, p_addr, cs, neg_m);
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&p_ready[wg]);
+        mbar_arrive(&p_ready[a]);
       }
+      pv_base += (uint32_t)n_it;
       // ------------------------------ epilogue ------------------------------
       mbar_wait(&tile_done, it & 1, ctx, 503);
       tc_fence_after();
-      sML[(wg * 2 + 0) * 128 + row] = m;
-      sML[(wg * 2 + 1) * 128 + row] = l;
+      float* xch = sX + 512;
+      xch[wg * 128 + row] = l;
       named_bar_sync(1, 256);
-      const float m0 = sML[0 * 128 + row], l0 = sML[1 * 128 + row];
-      const float m1 = sML[2 * 128 + row], l1 = sML[3 * 128 + row];
-      const float mm = fmaxf(m0, m1);
-      const float f0 = (m0 == -INFINITY) ? 0.f : ex2(m0 - mm);
-      const float f1 = (m1 == -INFINITY) ? 0.f : ex2(m1 - mm);
-      const float L = l0 * f0 + l1 * f1;
+      const float L = l + xch[(wg ^ 1) * 128 + row];
       const float inv = L > 0.f ? 1.0f / L : 0.f;
-      const bool have0 = n_it >= 1, have1 = n_it >= 2;
+      const bool have_o = n_it >= 1;
       const bool row_ok = row < sg.nrows;
       const size_t tok = (size_t)sg.q_tok0 + r / g;
       const int head = sg.h * g + r % g;
       __nv_bfloat16* orow = A.out + (tok * P.num_q_heads + head) * kHeadDim + wg * 64;
 #pragma unroll
       for (int k = 0; k < 2; ++k) {
-        uint32_t a0[32], a1[32];
-        if (have0) tmem_ld32(lane_base + 256 + wg * 64 + k * 32, a0);
-        if (have1) tmem_ld32(lane_base + 384 + wg * 64 + k * 32, a1);
-        tmem_wait_ld();
+        uint32_t a0[32];
+        if (have_o) {
+          tmem_ld32(o_addr + k * 32, a0);
+          tmem_wait_ld();
+        }
         uint32_t o[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          float v0 = 0.f, v1 = 0.f;
-          if (have0) {
-            v0 = __uint_as_float(a0[2 * j]) * f0;
-            v1 = __uint_as_float(a0[2 * j + 1]) * f0;
-          }
-          if (have1) {
-            v0 = fmaf(__uint_as_float(a1[2 * j]), f1, v0);
-            v1 = fmaf(__uint_as_float(a1[2 * j + 1]), f1, v1);
-          }
-          o[j] = pack_bf16x2(v0 * inv, v1 * inv);
+          const float v0 = have_o ? __uint_as_float(a0[2 * j]) * inv : 0.f;
+          const float v1 = have_o ? __uint_as_float(a0[2 * j + 1]) * inv : 0.f;
+          o[j] = pack_bf16x2(v0, v1);
         }
         if (row_ok) {
           uint4* dst = reinterpret_cast<uint4*>(orow + k * 32);
@@ -505,9 +507,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         }
       }
       if (wg == 0 && row_ok && A.lse != nullptr)
-        A.lse[(size_t)head * P.total_q + tok] = (mm + log2f(L)) * 0.6931471805599453f;
+        A.lse[(size_t)head * P.total_q + tok] = (m + log2f(L)) * 0.6931471805599453f;
       tc_fence_before();
-      named_bar_sync(1, 256);
+      named_bar_sync(1, 256);   // the exchange buffers are reused by the next tile
       mbar_arrive(&info_empty[slot]);
     }
   }
