@@ -130,6 +130,27 @@ fp2_status fp2_dense_prefill(fp2_plan* plan, const void* q, const void* k_cache,
                              const float* q_scale, const float* k_scale, const float* v_scale, void* out,
                              float* lse, void* workspace, fp2_stream stream);
 
+/* (No counterpart in the paper.)  fp2_dense_prefill for callers that have no device workspace to hand in and
+ * may not create one: a plug-in whose host passes it fixed input and output buffers and forbids device
+ * allocation, or code on a path where the memory allocator must not be entered (a framework callback, a
+ * latency-critical loop that may not take the allocator's lock).  The scratch
+ * of the dense path (status block, work counter, work order, counting-sort histogram) lives in a device array
+ * that is part of the library image: about 0.4 MB on every GPU that loads the library, held until exit.
+ *   - Limits: at most 65536 segments and 32 KV heads; larger plans are rejected with FP2_ERR_CAPACITY.
+ *     BF16 only, like fp2_dense_prefill.
+ *   - The call allocates and frees nothing.  The first call on a device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current); that first call should come before any stream
+ *     capture.
+ *   - All calls on a device share the one array, and it keeps what the previous call left: the entry point
+ *     clears the words that must start at zero, on `stream`.  Two calls whose kernels overlap on the GPU
+ *     (different streams, no dependency) race on it -- serialise them.
+ *   - The status block of this variant is internal; fp2_read_status does not see it.
+ * Arguments and results as fp2_dense_prefill, without `workspace`. */
+fp2_status fp2_dense_prefill_static(fp2_plan* plan, const void* q, const void* k_cache, const void* v_cache,
+                                    const int32_t* page_table, const int32_t* cu_seqlens_q,
+                                    const int32_t* seqlens_k, const float* q_scale, const float* k_scale,
+                                    const float* v_scale, void* out, float* lse, fp2_stream stream);
+
 /* Synchronises `stream`, reads the status block of `workspace` and clears it.  Returns FP2_ERR_TIMEOUT if a
  * bounded wait expired, FP2_ERR_INVALID_ARG if a list entry had to be clamped, else FP2_OK.  If
  * h_status_words is not NULL it receives the 8 raw int32 words (host memory). */

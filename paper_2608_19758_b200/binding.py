@@ -18,7 +18,7 @@ STATUS_NAMES = {0: "FP2_OK", 1: "FP2_ERR_INVALID_ARG", 2: "FP2_ERR_UNSUPPORTED",
                 4: "FP2_ERR_CUDA", 5: "FP2_ERR_TIMEOUT"}
 
 EXPORTS = ["fp2_plan_create", "fp2_plan_sizes", "fp2_plan_destroy", "fp2_plan_segment", "fp2_select_blocks",
-           "fp2_sparse_prefill", "fp2_dense_prefill", "fp2_read_status", "fp2_last_launch_count",
+           "fp2_sparse_prefill", "fp2_dense_prefill", "fp2_dense_prefill_static", "fp2_read_status", "fp2_last_launch_count",
            "fp2_status_string"]
 
 
@@ -71,6 +71,9 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.fp2_dense_prefill.argtypes = [C.c_void_p, vp, vp, vp, i32p, i32p, i32p, f32p, f32p, f32p, vp, f32p, vp,
                                       C.c_void_p]
     lib.fp2_dense_prefill.restype = C.c_int
+    lib.fp2_dense_prefill_static.argtypes = [C.c_void_p, vp, vp, vp, i32p, i32p, i32p, f32p, f32p, f32p, vp, f32p,
+                                             C.c_void_p]
+    lib.fp2_dense_prefill_static.restype = C.c_int
     lib.fp2_read_status.argtypes = [C.c_void_p, vp, C.POINTER(C.c_int32), C.c_void_p]
     lib.fp2_read_status.restype = C.c_int
     lib.fp2_last_launch_count.argtypes = [C.c_void_p]
@@ -179,6 +182,15 @@ def fp2_dense_prefill(plan: Plan, q, k_cache, v_cache, page_table, cu_seqlens_q,
                                     _ptr(cu_seqlens_q), _ptr(seqlens_k), _ptr(q_scale), _ptr(k_scale),
                                     _ptr(v_scale), _ptr(out), _ptr(lse), _ptr(workspace), _stream(stream)),
            "fp2_dense_prefill")
+
+
+def fp2_dense_prefill_static(plan: Plan, q, k_cache, v_cache, page_table, cu_seqlens_q, seqlens_k, q_scale, k_scale,
+                             v_scale, out, lse, stream=None):
+    """Dense prefill without a caller workspace: the library's built-in device scratch is used."""
+    _check(load().fp2_dense_prefill_static(plan.handle, _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(page_table),
+                                           _ptr(cu_seqlens_q), _ptr(seqlens_k), _ptr(q_scale), _ptr(k_scale),
+                                           _ptr(v_scale), _ptr(out), _ptr(lse), _stream(stream)),
+           "fp2_dense_prefill_static")
 
 
 def fp2_read_status(plan: Plan, workspace, stream=None, raise_on_error: bool = True):

@@ -385,6 +385,88 @@ extern "C" fp2_status fp2_dense_prefill(fp2_plan* pl, const void* q, const void*
   return run_attention(pl, q, k, v, pt, cu, lk, nullptr, nullptr, qs, ks, vs, out, lse, workspace, false, stream);
 }
 
+// ------------------------------------------------------------------------------------------------------
+// Dense prefill for callers that cannot provide a workspace (see include/fp2.h).  The scratch the dense path
+// needs -- status block, work counter, work order, histogram of the counting sort -- lives in a file-scope
+// device array instead of caller memory.  Nothing here allocates.
+// ------------------------------------------------------------------------------------------------------
+constexpr int kStaticMaxSegments = 65536;
+constexpr int kStaticMaxKvHeads = 32;
+constexpr size_t kStaticOffOrder = 1024;
+constexpr size_t kStaticOffHist = kStaticOffOrder + sizeof(int32_t) * kStaticMaxSegments;
+constexpr size_t kStaticBytes = kStaticOffHist + sizeof(int32_t) * ((size_t)kStaticMaxKvHeads * kCountBuckets + 256);
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+// In host code `g_static_scratch` is only a handle; the device address comes from cudaGetSymbolAddress,
+// asked once per device with that device current.
+constexpr int kMaxDevices = 64;
+static unsigned char* g_static_ptr[kMaxDevices];
+
+static fp2_status static_scratch_for(int device, unsigned char** out) {
+  if (device < 0 || device >= kMaxDevices) return FP2_ERR_UNSUPPORTED;
+  if (!g_static_ptr[device]) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return FP2_ERR_CUDA;
+    g_static_ptr[device] = reinterpret_cast<unsigned char*>(ptr);
+  }
+  *out = g_static_ptr[device];
+  return FP2_OK;
+}
+
+extern "C" fp2_status fp2_dense_prefill_static(fp2_plan* pl, const void* q, const void* k, const void* v,
+                                               const int32_t* pt, const int32_t* cu, const int32_t* lk,
+                                               const float* qs, const float* ks, const float* vs, void* out,
+                                               float* lse, fp2_stream stream) {
+  if (!pl || !q || !k || !v || !pt || !cu || !lk || !out) return FP2_ERR_INVALID_ARG;
+  if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out, 16)) return FP2_ERR_INVALID_ARG;
+  if (pl->device < 0) return FP2_ERR_CUDA;
+  if (pl->dev.fp8) return FP2_ERR_UNSUPPORTED;
+  if (pl->nseg > kStaticMaxSegments || pl->prm.num_kv_heads > kStaticMaxKvHeads) return FP2_ERR_CAPACITY;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FP2_ERR_CUDA;
+  if (dev != pl->device) return FP2_ERR_INVALID_ARG;
+  fp2_status s = set_attrs(pl);
+  if (s != FP2_OK) return s;
+  unsigned char* sw = nullptr;
+  if ((s = static_scratch_for(dev, &sw)) != FP2_OK) return s;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  pl->last_launches = 0;
+  if (pl->nseg == 0) return FP2_OK;
+  const int nseg = (int)pl->nseg;
+  int32_t* order = reinterpret_cast<int32_t*>(sw + kStaticOffOrder);
+  int32_t* hist = reinterpret_cast<int32_t*>(sw + kStaticOffHist);
+  const int nb = pl->prm.num_kv_heads * kCountBuckets;
+  // the array keeps the previous call's contents: status, counter and histogram must start at zero
+  if (cudaMemsetAsync(sw, 0, 1024, st) != cudaSuccess) return FP2_ERR_CUDA;
+  if (cudaMemsetAsync(hist, 0, sizeof(int32_t) * (size_t)(nb + 1), st) != cudaSuccess) return FP2_ERR_CUDA;
+  const int blocks = (nseg + 255) / 256;
+  order_hist_kernel<<<blocks, 256, 0, st>>>(pl->d_segs, nullptr, nseg, hist);
+  order_scan_kernel<<<1, 1024, 0, st>>>(hist, nb);
+  order_scatter_kernel<<<blocks, 256, 0, st>>>(pl->d_segs, nullptr, nseg, hist, order);
+  const int64_t slots = (int64_t)pl->prm.num_pages * pl->prm.page_size;
+  CUtensorMap mk, mv;
+  if (!make_map(pl, &mk, k, slots, pl->prm.num_kv_heads, pl->prm.page_size, false) ||
+      !make_map(pl, &mv, v, slots, pl->prm.num_kv_heads, pl->prm.page_size, false))
+    return FP2_ERR_CUDA;
+  AttnArgs a;
+  a.q = reinterpret_cast<const uint8_t*>(q);
+  a.page_table = pt;
+  a.segs = pl->d_segs;
+  a.order = order;
+  a.seg_count = nullptr;
+  a.blk_idx = nullptr;
+  a.q_scale = qs; a.k_scale = ks; a.v_scale = vs;
+  a.out = reinterpret_cast<__nv_bfloat16*>(out);
+  a.lse = lse;
+  a.work_counter = reinterpret_cast<int*>(sw + 64);
+  a.status = reinterpret_cast<int*>(sw);
+  const unsigned grid = (unsigned)(pl->nseg < pl->num_sms ? pl->nseg : pl->num_sms);
+  // the dense path stages no pooled chunks: the two pooled-mean maps are never dereferenced
+  sparse_attn_kernel<false><<<grid, kAttnThreads, kAttnSmemBytes, st>>>(mk, mv, mk, mv, a, pl->dev);
+  pl->last_launches = 4;
+  return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
+}
+
 extern "C" fp2_status fp2_read_status(fp2_plan* pl, void* workspace, int32_t* h_words, fp2_stream stream) {
   if (!pl || !workspace) return FP2_ERR_INVALID_ARG;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
