@@ -22,8 +22,9 @@ struct SegInfo {
   int32_t J_lo;     // block of the first row's absolute position
   int32_t J_hi;     // block of the last row's absolute position (candidates are 0..J_hi)
   int32_t blk_off;  // first row of this sequence in the pooled-mean arrays
-  int32_t pad;
+  int32_t seg;      // index of this segment in segment order
   int64_t off;      // seg_offset: start of this segment's list in blk_idx
+  __host__ __device__ int h_seg() const { return seg; }
 };
 static_assert(sizeof(SegInfo) == 56, "SegInfo layout");
 

@@ -78,7 +78,8 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
     ntiles_tot += (g * lq + kTileRows - 1) / kTileRows;
     nblk_tot += nblk;
   }
-  if (ntiles_tot * p->num_kv_heads > (int64_t)0x7fffffff || nblk_tot > (int64_t)0x7fffffff) return FP2_ERR_CAPACITY;
+  if (ntiles_tot * p->num_kv_heads > (int64_t)0x7fffffff || nblk_tot * p->num_kv_heads > (int64_t)0x7fffffff)
+    return FP2_ERR_CAPACITY;
 
   fp2_plan* pl = new (std::nothrow) fp2_plan();
   if (!pl) return FP2_ERR_CUDA;
@@ -113,7 +114,7 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
         s.J_lo = (int)((pre + r0 / g) / kBlock);
         s.J_hi = (int)((pre + (r1 - 1) / g) / kBlock);
         s.blk_off = (int32_t)boff;
-        s.pad = 0;
+        s.seg = (int32_t)(p->num_kv_heads * tile_off + (int64_t)h * nt + t);
         s.off = 0;
       }
     tile_off += nt;
@@ -265,7 +266,7 @@ static fp2_status check_common(fp2_plan* pl, const void* q, const void* k, const
 static fp2_status launch_pool(fp2_plan* pl, const void* k, const void* v, const int32_t* pt, const int32_t* lk,
                               const float* ks, const float* vs, uint8_t* ws, cudaStream_t st) {
   if (pl->nblk_tot == 0) return FP2_OK;
-  dim3 grid((unsigned)pl->nblk_tot, (unsigned)pl->prm.num_kv_heads);
+  const unsigned grid = (unsigned)(pl->nblk_tot * pl->prm.num_kv_heads);
   __nv_bfloat16* khi = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_khi);
   __nv_bfloat16* klo = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_klo);
   __nv_bfloat16* vb = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_vbar);
@@ -315,12 +316,15 @@ extern "C" fp2_status fp2_select_blocks(fp2_plan* pl, const void* q, const void*
       !make_map(pl, &mlo, ws + pl->ws_klo, pl->nblk_tot, pl->prm.num_kv_heads, 128, false))
     return FP2_ERR_CUDA;
   int* status = reinterpret_cast<int*>(ws + pl->ws_status);
+  int* counter = reinterpret_cast<int*>(ws + pl->ws_counter) + 4;   // the attention kernel uses word 0
+  if (cudaMemsetAsync(counter, 0, sizeof(int), st) != cudaSuccess) return FP2_ERR_CUDA;
+  const unsigned grid = (unsigned)(pl->nseg < pl->num_sms ? pl->nseg : pl->num_sms);
   if (pl->dev.fp8)
-    score_select_kernel<true><<<(unsigned)pl->nseg, kScoreThreads, kScoreSmemBytes, st>>>(
-        mhi, mlo, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, status);
+    score_select_kernel<true><<<grid, kScoreThreads, kScoreSmemBytes, st>>>(
+        mhi, mlo, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, counter, status);
   else
-    score_select_kernel<false><<<(unsigned)pl->nseg, kScoreThreads, kScoreSmemBytes, st>>>(
-        mhi, mlo, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, status);
+    score_select_kernel<false><<<grid, kScoreThreads, kScoreSmemBytes, st>>>(
+        mhi, mlo, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, counter, status);
   pl->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }

@@ -35,7 +35,8 @@ __device__ __forceinline__ void accum16(const uint4& v, float* acc) {
   }
 }
 
-// grid (nblk_tot, Hkv), 256 threads.
+// 1-D grid of nblk_tot * Hkv CTAs, KV head fastest: CTAs that run together read neighbouring heads of the same
+// tokens, i.e. whole contiguous token rows of the cache.  256 threads.
 template <bool FP8>
 __global__ void __launch_bounds__(256) pool_kv_kernel(const uint8_t* __restrict__ k_cache,
                                                       const uint8_t* __restrict__ v_cache,
@@ -55,7 +56,7 @@ __global__ void __launch_bounds__(256) pool_kv_kernel(const uint8_t* __restrict_
 
   __shared__ float red[2][ROWS_PER_PASS][kHeadDim + 4];
 
-  const int gblk = blockIdx.x, h = blockIdx.y;
+  const int gblk = blockIdx.x / P.num_kv_heads, h = blockIdx.x % P.num_kv_heads;
   // sequence of this pooled block: binary search in blk_off
   int lo = 0, hi = P.num_seqs;
   while (hi - lo > 1) {

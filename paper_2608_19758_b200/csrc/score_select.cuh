@@ -1,4 +1,5 @@
-// Fused block scoring and selection (Eq. 19, Eq. 20; Algorithm 1 lines 3-5), one CTA per segment.
+// Fused block scoring and selection (Eq. 19, Eq. 20; Algorithm 1 lines 3-5); persistent, one CTA per SM,
+// segments handed out heaviest first through a global counter.
 //
 // For the packed query tile I (128 rows of one KV head) and every candidate block J <= J_hi:
 //     s_iJ = scale * q_i . kbar_J,   m_J = max_i s_iJ,   S_J = sum_i 2^{(s_iJ - m_J) log2 e}
@@ -12,8 +13,10 @@
 // BF16 (hi, lo) pair accumulated into the same fp32 accumulator, which keeps the energies accurate to ~1e-5
 // relative; a single BF16 kbar would move them by ~3e-3 and flip list entries.
 //
-// Roles: warps 0-3 / 4-7 = two consumer warpgroups alternating over chunks (TMEM accumulators 0 / 1),
-// warp 8 = TMA producer of kbar chunks, warp 9 = UMMA issuer.
+// Roles: warps 0-3 / 4-7 = two consumer warpgroups alternating over chunks (TMEM accumulators 0 / 1) and doing
+// the selection of their tile together; warp 8 = TMA producer of kbar pieces; warp 9 = UMMA issuer; warps 10-11
+// fetch the next segment and stage its query tile into the free one of two Q buffers, so that the next tile's
+// MMAs start while the current tile is still being exponentiated and selected.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
@@ -22,9 +25,9 @@
 
 namespace fp2 {
 
-constexpr int kScoreThreads = 320;
-constexpr int kScoreStageBytes = 65536;  // kbar_hi chunk (32 KB) + kbar_lo chunk (32 KB)
-constexpr int kScoreSmemBytes = 1024 /*align*/ + 32768 /*Q*/ + 2 * kScoreStageBytes + 2 * kMaxBlocks * 4 + 1024;
+constexpr int kScoreThreads = 384;
+constexpr int kScoreStages = 3;          // ring of 32 KB pieces: the kbar_hi or the kbar_lo half of a 128-block chunk
+constexpr int kScoreSmemBytes = 1024 /*align*/ + 2 * 32768 /*Q x2*/ + kScoreStages * 32768 + 2 * kMaxBlocks * 4 + 1024;
 
 // Query tile -> shared memory in the K-major 128-byte-swizzled layout the UMMA descriptors expect:
 // BF16: two 64-column halves of [128 rows x 128 B]; FP8 is widened to BF16 on the way (exact).
@@ -104,41 +107,68 @@ __device__ __forceinline__ void score_chunk(uint32_t lane_addr, float cs, const 
   sum_out = ((s8[0] + s8[1]) + (s8[2] + s8[3])) + ((s8[4] + s8[5]) + (s8[6] + s8[7]));
 }
 
+// BF16 query tile -> shared memory with cp.async: every 16-byte piece of the tile is in flight at once (the
+// register-staged variant above keeps only a few loads per thread in flight and was latency-bound at one tile
+// per ~12 us).  Same layout and zero fill as load_q_tile_bf16; returns after the copies have landed.
+__device__ __forceinline__ void load_q_tile_async(uint8_t* sQ, const uint8_t* __restrict__ q, const SegInfo& sg,
+                                                  const DevParams& P, int t, int nthr) {
+  const int g = P.group;
+  const uint32_t base = smem_u32(sQ);
+  for (int i = t; i < kTileRows * 16; i += nthr) {
+    const int row = i >> 4, ch = i & 15;
+    const uint8_t* src = q;
+    uint32_t nbytes = 0;
+    if (row < sg.nrows) {
+      const int r = sg.r0 + row;
+      const size_t tok = (size_t)sg.q_tok0 + r / g;
+      const size_t head = (size_t)sg.h * g + r % g;
+      src = q + ((tok * P.num_q_heads + head) * kHeadDim + ch * 8) * 2;
+      nbytes = 16;
+    }
+    cp_async16(base + (ch >> 3) * 16384 + sw128_offset(row, ch & 7), src, nbytes);
+  }
+  cp_async_wait_all();
+}
+
 template <bool FP8>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_constant__ CUtensorMap map_klo,
                     const uint8_t* __restrict__ q, const SegInfo* __restrict__ segs, const float* __restrict__ q_scale,
                     DevParams P, int64_t* __restrict__ seg_offset, int32_t* __restrict__ seg_count,
-                    int32_t* __restrict__ blk_idx, int* __restrict__ status) {
+                    int32_t* __restrict__ blk_idx, int* __restrict__ work_counter, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem;
-  uint8_t* sStage = smem + 32768;
-  float* sS = reinterpret_cast<float*>(sStage + 2 * kScoreStageBytes);  // per candidate: S_J, later E_J
+  uint8_t* sQ = smem;                                    // 2 x 32 KB query tiles
+  uint8_t* sStage = smem + 2 * 32768;                    // kScoreStages x 32 KB pieces (kbar_hi or kbar_lo chunk)
+  float* sS = reinterpret_cast<float*>(sStage + kScoreStages * 32768);  // per candidate: S_J, later E_J
   float* sM = sS + kMaxBlocks;                                          // per candidate: m_J
-  float* sC = sM + kMaxBlocks;                                          // per tile row: logit multiplier (FP8)
+  float* sC = sM + kMaxBlocks;                                          // [2][128] per-row logit multiplier (FP8)
 
-  __shared__ uint64_t full[2], empty[2], acc_full[2], acc_empty[2];
+  __shared__ SegInfo info[2];
+  __shared__ int info_valid[2];
+  __shared__ uint64_t info_full[2], info_empty[2], q_full[2], q_empty[2];
+  __shared__ uint64_t full[kScoreStages], empty[kScoreStages], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
   __shared__ float red[8];
   __shared__ int wsum[8];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  // heaviest tiles (largest candidate count) of every sequence come last in segment order: launch them first
-  const int seg = P.nseg - 1 - (int)blockIdx.x;
-  const SegInfo sg = segs[seg];
-  const int ncand = sg.J_hi + 1;
-  const int nchunks = (ncand + 127) >> 7;
   WaitCtx ctx{status, &abort_flag};
 
   if (tid == 0) {
     abort_flag = 0;
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&full[i], 1);
-      mbar_init(&empty[i], 1);
+      mbar_init(&info_full[i], 1);
+      mbar_init(&info_empty[i], 2 + 256);
+      mbar_init(&q_full[i], 64);
+      mbar_init(&q_empty[i], 1);
       mbar_init(&acc_full[i], 1);
       mbar_init(&acc_empty[i], 128);
+    }
+    for (int i = 0; i < kScoreStages; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], 1);
     }
     fence_barrier_init();
   }
@@ -146,132 +176,183 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
     tmem_alloc(&tmem_base_s, 256);
     tmem_relinquish();
   }
-  if (warp < 8) {
-    load_q_tile_bf16<FP8>(sQ, q, sg, P, tid, 256);
-    if constexpr (FP8) {
-      if (tid < kTileRows) {
-        const int r = sg.r0 + tid;
-        sC[tid] = P.scale_log2 * q_scale[sg.h * P.group + r % P.group];
-      }
-    }
-    fence_proxy_async();
-  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
 
-  if (warp == 8) {
-    // ---------------- producer: kbar chunks (hi and lo) via TMA ----------------
+  if (warp >= 10) {
+    // ---------------- set-up: next segment (heaviest first), query tile into the free Q buffer ----------------
+    const int t64 = tid - 320;
+    for (int it = 0;; ++it) {
+      const int slot = it & 1;
+      if (it >= 2) mbar_wait(&info_empty[slot], ((it >> 1) - 1) & 1, ctx, 111);
+      if (t64 == 0) {
+        const int w = atomicAdd(work_counter, 1);
+        info_valid[slot] = w < P.nseg;
+        if (w < P.nseg) info[slot] = segs[P.nseg - 1 - w];
+      }
+      named_bar_sync(2, 64);
+      const bool valid = info_valid[slot] != 0;
+      if (t64 == 0) mbar_arrive(&info_full[slot]);
+      if (!valid) break;
+      const SegInfo sg = info[slot];
+      if (it >= 2) mbar_wait(&q_empty[slot], ((it >> 1) - 1) & 1, ctx, 112);
+      if constexpr (FP8) load_q_tile_bf16<true, 8>(sQ + slot * 32768, q, sg, P, t64, 64);
+      else load_q_tile_async(sQ + slot * 32768, q, sg, P, t64, 64);
+      if constexpr (FP8) {
+        for (int j = t64; j < kTileRows; j += 64)
+          sC[slot * 128 + j] = P.scale_log2 * q_scale[sg.h * P.group + (sg.r0 + j) % P.group];
+      }
+      fence_proxy_async();
+      mbar_arrive(&q_full[slot]);
+    }
+  } else if (warp == 8) {
+    // ---------------- producer: kbar pieces (hi, lo of every 128-block chunk) via TMA ----------------
     if (lane == 0) {
       tma_prefetch_desc(&map_khi);
       tma_prefetch_desc(&map_klo);
-      for (int c = 0; c < nchunks; ++c) {
-        const int s = c & 1;
-        if (c >= 2) mbar_wait(&empty[s], ((c >> 1) - 1) & 1, ctx, 101);
-        uint8_t* dst = sStage + s * kScoreStageBytes;
-        mbar_arrive_expect_tx(&full[s], kScoreStageBytes);
-        const int row0 = sg.blk_off + c * 128;
-        tma_load_3d(dst, &map_khi, &full[s], 0, sg.h, row0);
-        tma_load_3d(dst + 16384, &map_khi, &full[s], 64, sg.h, row0);
-        tma_load_3d(dst + 32768, &map_klo, &full[s], 0, sg.h, row0);
-        tma_load_3d(dst + 49152, &map_klo, &full[s], 64, sg.h, row0);
+      uint32_t pc = 0;
+      for (int it = 0;; ++it) {
+        const int slot = it & 1;
+        mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 121);
+        if (!info_valid[slot]) break;
+        const int h = info[slot].h, blk_off = info[slot].blk_off;
+        const int nchunks = (info[slot].J_hi + 128) >> 7;
+        for (int c = 0; c < nchunks; ++c) {
+#pragma unroll
+          for (int part = 0; part < 2; ++part, ++pc) {
+            const int s = pc % kScoreStages;
+            if (pc >= kScoreStages) mbar_wait(&empty[s], ((pc / kScoreStages) - 1) & 1, ctx, 122);
+            uint8_t* dst = sStage + s * 32768;
+            mbar_arrive_expect_tx(&full[s], 32768);
+            const CUtensorMap* mp = part ? &map_klo : &map_khi;
+            tma_load_3d(dst, mp, &full[s], 0, h, blk_off + c * 128);
+            tma_load_3d(dst + 16384, mp, &full[s], 64, h, blk_off + c * 128);
+          }
+        }
+        mbar_arrive(&info_empty[slot]);
       }
     }
   } else if (warp == 9) {
-    // ---------------- UMMA issuer: acc[c&1] = kbar_hi Q^T + kbar_lo Q^T ----------------
+    // ---------------- UMMA issuer: acc[c & 1] = kbar_hi Q^T + kbar_lo Q^T ----------------
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(128, 128, 1, 1, 0, 0);
-      const uint32_t q_addr = smem_u32(sQ);
-      for (int c = 0; c < nchunks; ++c) {
-        const int s = c & 1;
-        mbar_wait(&full[s], (c >> 1) & 1, ctx, 102);
-        if (c >= 2) mbar_wait(&acc_empty[s], ((c >> 1) - 1) & 1, ctx, 103);
-        tc_fence_after();
-        const uint32_t a_addr = smem_u32(sStage + s * kScoreStageBytes);
+      uint32_t pc = 0, ac0 = 0, ac1 = 0;
+      for (int it = 0;; ++it) {
+        const int slot = it & 1;
+        mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 131);
+        if (!info_valid[slot]) break;
+        const int nchunks = (info[slot].J_hi + 128) >> 7;
+        mbar_wait(&q_full[slot], (it >> 1) & 1, ctx, 132);
+        const uint32_t q_addr = smem_u32(sQ + slot * 32768);
+        for (int c = 0; c < nchunks; ++c) {
+          const int a = c & 1;
+          uint32_t& ac = a ? ac1 : ac0;
+          if (ac >= 1) mbar_wait(&acc_empty[a], (ac - 1) & 1, ctx, 133);
+          ++ac;
 #pragma unroll
-        for (int part = 0; part < 2; ++part) {
+          for (int part = 0; part < 2; ++part, ++pc) {
+            const int s = pc % kScoreStages;
+            mbar_wait(&full[s], (pc / kScoreStages) & 1, ctx, 134);
+            tc_fence_after();
+            const uint32_t a_addr = smem_u32(sStage + s * 32768);
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
-            const uint64_t ad = make_smem_desc_sw128(a_addr + part * 32768 + off, 16, 1024);
-            const uint64_t bd = make_smem_desc_sw128(q_addr + off, 16, 1024);
-            umma_f16_ss(tmem + s * 128, ad, bd, idesc, (part | ks) != 0);
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+              const uint64_t ad = make_smem_desc_sw128(a_addr + off, 16, 1024);
+              const uint64_t bd = make_smem_desc_sw128(q_addr + off, 16, 1024);
+              umma_f16_ss(tmem + a * 128, ad, bd, idesc, (part | ks) != 0);
+            }
+            umma_commit(&empty[s]);
           }
+          umma_commit(&acc_full[a]);
         }
-        umma_commit(&empty[s]);
-        umma_commit(&acc_full[s]);
+        umma_commit(&q_empty[slot]);
+        mbar_arrive(&info_empty[slot]);
       }
     }
   } else {
-    // ---------------- consumers: per pooled key, max and exp-sum over the tile's rows ----------------
+    // ---------------- consumers: per pooled key, max and exp-sum over the tile's rows; then selection ----------------
     const int wg = warp >> 2;
     const int key = (warp & 3) * 32 + lane;  // TMEM lane = pooled key within the chunk
     const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + wg * 128;
     const float cs = P.scale_log2;
-    for (int c = wg; c < nchunks; c += 2) {
-      mbar_wait(&acc_full[wg], (c >> 1) & 1, ctx, 104);
-      tc_fence_after();
-      float m, sum;
-      if (sg.nrows == kTileRows) score_chunk<FP8, false>(lane_addr, cs, sC, kTileRows, &acc_empty[wg], m, sum);
-      else score_chunk<FP8, true>(lane_addr, cs, sC, sg.nrows, &acc_empty[wg], m, sum);
-      const int J = c * 128 + key;
-      if (J < ncand) {
-        sS[J] = sum;
-        sM[J] = m;
+    uint32_t uc = 0;  // uses of this warpgroup's accumulator
+    for (int it = 0;; ++it) {
+      const int slot = it & 1;
+      mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 141);
+      if (!info_valid[slot]) break;
+      const SegInfo sg = info[slot];
+      const int seg = sg.h_seg();
+      const int ncand = sg.J_hi + 1;
+      const int nchunks = (ncand + 127) >> 7;
+      for (int c = wg; c < nchunks; c += 2, ++uc) {
+        mbar_wait(&acc_full[wg], uc & 1, ctx, 142);
+        tc_fence_after();
+        float m, sum;
+        if (sg.nrows == kTileRows) score_chunk<FP8, false>(lane_addr, cs, sC + slot * 128, kTileRows, &acc_empty[wg], m, sum);
+        else score_chunk<FP8, true>(lane_addr, cs, sC + slot * 128, sg.nrows, &acc_empty[wg], m, sum);
+        const int J = c * 128 + key;
+        if (J < ncand) {
+          sS[J] = sum;
+          sM[J] = m;
+        }
       }
-    }
-    // ---------------- selection: all 256 consumer threads ----------------
-    named_bar_sync(1, 256);
-    float lm = -INFINITY;
-    for (int J = tid; J < ncand; J += 256) lm = fmaxf(lm, sM[J]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) lm = fmaxf(lm, __shfl_xor_sync(0xffffffffu, lm, o));
-    if (lane == 0) red[warp] = lm;
-    named_bar_sync(1, 256);
-    float M = red[0];
-#pragma unroll
-    for (int i = 1; i < 8; ++i) M = fmaxf(M, red[i]);
-    named_bar_sync(1, 256);
-    float le = 0.f;
-    for (int J = tid; J < ncand; J += 256) {
-      const float e = sS[J] * exp2f(sM[J] - M);
-      sS[J] = e;
-      le = fmaxf(le, e);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) le = fmaxf(le, __shfl_xor_sync(0xffffffffu, le, o));
-    if (lane == 0) red[warp] = le;
-    named_bar_sync(1, 256);
-    float maxE = red[0];
-#pragma unroll
-    for (int i = 1; i < 8; ++i) maxE = fmaxf(maxE, red[i]);
-    const float thr = P.alpha * maxE;
-    const int win_lo = sg.J_lo - P.window_blocks;
-    int base = 0;
-    for (int J0 = 0; J0 < ncand; J0 += 256) {
-      const int J = J0 + tid;
-      const bool keep = J < ncand && (sS[J] >= thr || J < P.sink_blocks || J >= win_lo);
-      const unsigned bal = __ballot_sync(0xffffffffu, keep);
-      if (lane == 0) wsum[warp] = __popc(bal);
+      // ---------------- selection: all 256 consumer threads ----------------
       named_bar_sync(1, 256);
-      int before = 0, total = 0;
+      float lm = -INFINITY;
+      for (int J = tid; J < ncand; J += 256) lm = fmaxf(lm, sM[J]);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int v = wsum[i];
-        before += (i < warp) ? v : 0;
-        total += v;
+      for (int o = 16; o > 0; o >>= 1) lm = fmaxf(lm, __shfl_xor_sync(0xffffffffu, lm, o));
+      if (lane == 0) red[warp] = lm;
+      named_bar_sync(1, 256);
+      float M = red[0];
+#pragma unroll
+      for (int i = 1; i < 8; ++i) M = fmaxf(M, red[i]);
+      named_bar_sync(1, 256);
+      float le = 0.f;
+      for (int J = tid; J < ncand; J += 256) {
+        const float e = sS[J] * exp2f(sM[J] - M);
+        sS[J] = e;
+        le = fmaxf(le, e);
       }
-      if (keep) blk_idx[sg.off + base + before + __popc(bal & ((1u << lane) - 1u))] = J;
-      base += total;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) le = fmaxf(le, __shfl_xor_sync(0xffffffffu, le, o));
+      if (lane == 0) red[warp] = le;
       named_bar_sync(1, 256);
-    }
-    if (tid == 0) {
-      seg_count[seg] = base;
-      seg_offset[seg] = sg.off;
-      if (seg == P.nseg - 1) seg_offset[P.nseg] = sg.off + ncand;
+      float maxE = red[0];
+#pragma unroll
+      for (int i = 1; i < 8; ++i) maxE = fmaxf(maxE, red[i]);
+      const float thr = P.alpha * maxE;
+      const int win_lo = sg.J_lo - P.window_blocks;
+      int base = 0;
+      for (int J0 = 0; J0 < ncand; J0 += 256) {
+        const int J = J0 + tid;
+        const bool keep = J < ncand && (sS[J] >= thr || J < P.sink_blocks || J >= win_lo);
+        const unsigned bal = __ballot_sync(0xffffffffu, keep);
+        if (lane == 0) wsum[warp] = __popc(bal);
+        named_bar_sync(1, 256);
+        int before = 0, total = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int v = wsum[i];
+          before += (i < warp) ? v : 0;
+          total += v;
+        }
+        if (keep) blk_idx[sg.off + base + before + __popc(bal & ((1u << lane) - 1u))] = J;
+        base += total;
+        named_bar_sync(1, 256);
+      }
+      if (tid == 0) {
+        seg_count[seg] = base;
+        seg_offset[seg] = sg.off;
+        if (seg == P.nseg - 1) seg_offset[P.nseg] = sg.off + ncand;
+      }
+      mbar_arrive(&info_empty[slot]);
     }
   }
+  if (abort_flag) __nanosleep(2000000);
   tc_fence_before();
   __syncthreads();
   if (warp == 9) tmem_dealloc(tmem, 256);

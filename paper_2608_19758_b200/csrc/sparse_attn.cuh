@@ -249,7 +249,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       if (!valid) break;
       // Q tile: wait until every S = Q K^T of the previous unit has completed, then overwrite
       if (it >= 1) mbar_wait(&q_empty, (it - 1) & 1, ctx, 202);
-      load_q_tile_bf16<FP8, 4>(sQ, A.q, ti.sg, P, t64, 64);
+      load_q_tile_async(sQ, A.q, ti.sg, P, t64, 64);
       fence_proxy_async();
       mbar_arrive(&q_full);
     }
