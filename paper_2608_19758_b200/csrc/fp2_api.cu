@@ -316,15 +316,13 @@ extern "C" fp2_status fp2_select_blocks(fp2_plan* pl, const void* q, const void*
       !make_map(pl, &mlo, ws + pl->ws_klo, pl->nblk_tot, pl->prm.num_kv_heads, 128, false))
     return FP2_ERR_CUDA;
   int* status = reinterpret_cast<int*>(ws + pl->ws_status);
-  int* counter = reinterpret_cast<int*>(ws + pl->ws_counter) + 4;   // the attention kernel uses word 0
-  if (cudaMemsetAsync(counter, 0, sizeof(int), st) != cudaSuccess) return FP2_ERR_CUDA;
   const unsigned grid = (unsigned)(pl->nseg < pl->num_sms ? pl->nseg : pl->num_sms);
   if (pl->dev.fp8)
     score_select_kernel<true><<<grid, kScoreThreads, kScoreSmemBytes, st>>>(
-        mhi, mlo, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, counter, status);
+        mhi, mlo, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, status);
   else
     score_select_kernel<false><<<grid, kScoreThreads, kScoreSmemBytes, st>>>(
-        mhi, mlo, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, counter, status);
+        mhi, mlo, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, status);
   pl->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }

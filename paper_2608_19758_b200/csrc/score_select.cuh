@@ -1,11 +1,11 @@
 // Fused block scoring and selection (Eq. 19, Eq. 20; Algorithm 1 lines 3-5); persistent, one CTA per SM,
-// segments handed out heaviest first through a global counter.
+// segments dealt round-robin in heaviest-first order.
 //
 // For the packed query tile I (128 rows of one KV head) and every candidate block J <= J_hi:
 //     s_iJ = scale * q_i . kbar_J,   m_J = max_i s_iJ,   S_J = sum_i 2^{(s_iJ - m_J) log2 e}
-// (the per-block max / sum of Eq. 1), then  M = max_J m_J,  E_J = S_J 2^{(m_J - M) log2 e}  (the global
-// rescale of Eq. 2 / Eq. 20), threshold alpha * max_J E_J, forced sink / window / diagonal blocks, and an
-// ordered compaction of the survivors into the segment's list.
+// (the per-block max / sum of Eq. 1), then the energy in the log domain  e_J = m_J log2 e + log2 S_J  (the
+// global rescale of Eq. 2 / Eq. 20 only adds a constant), threshold  e_J >= log2 alpha + max_J e_J, forced
+// sink / window / diagonal blocks, and an ordered compaction of the survivors into the segment's list.
 //
 // The contraction runs on the tensor cores TRANSPOSED: A = a chunk of 128 pooled keys (rows = TMEM lanes),
 // B = the query tile (columns), so that each consumer thread owns one pooled key and the sum over the tile's
@@ -26,8 +26,11 @@
 namespace fp2 {
 
 constexpr int kScoreThreads = 384;
+constexpr int kScoreInfoSlots = 4;       // segment descriptors in flight
+constexpr int kScoreQBufs = 3;           // query tiles in flight: two loading while one is multiplied (one tile in
+                                         // flight per SM cannot cover the HBM latency-bandwidth product)
 constexpr int kScoreStages = 3;          // ring of 32 KB pieces: the kbar_hi or the kbar_lo half of a 128-block chunk
-constexpr int kScoreSmemBytes = 1024 /*align*/ + 2 * 32768 /*Q x2*/ + kScoreStages * 32768 + 2 * kMaxBlocks * 4 + 1024;
+constexpr int kScoreSmemBytes = 1024 /*align*/ + kScoreQBufs * 32768 + kScoreStages * 32768 + kMaxBlocks * 4 + 2048;
 
 // Query tile -> shared memory in the K-major 128-byte-swizzled layout the UMMA descriptors expect:
 // BF16: two 64-column halves of [128 rows x 128 B]; FP8 is widened to BF16 on the way (exact).
@@ -109,9 +112,10 @@ __device__ __forceinline__ void score_chunk(uint32_t lane_addr, float cs, const 
 
 // BF16 query tile -> shared memory with cp.async: every 16-byte piece of the tile is in flight at once (the
 // register-staged variant above keeps only a few loads per thread in flight and was latency-bound at one tile
-// per ~12 us).  Same layout and zero fill as load_q_tile_bf16; returns after the copies have landed.
+// per ~12 us).  Same layout and zero fill as load_q_tile_bf16; with `wait` it returns after the copies have landed,
+// otherwise the caller closes a cp.async group and waits for it later.
 __device__ __forceinline__ void load_q_tile_async(uint8_t* sQ, const uint8_t* __restrict__ q, const SegInfo& sg,
-                                                  const DevParams& P, int t, int nthr) {
+                                                  const DevParams& P, int t, int nthr, bool wait = true) {
   const int g = P.group;
   const uint32_t base = smem_u32(sQ);
   for (int i = t; i < kTileRows * 16; i += nthr) {
@@ -127,7 +131,7 @@ __device__ __forceinline__ void load_q_tile_async(uint8_t* sQ, const uint8_t* __
     }
     cp_async16(base + (ch >> 3) * 16384 + sw128_offset(row, ch & 7), src, nbytes);
   }
-  cp_async_wait_all();
+  if (wait) cp_async_wait_all();
 }
 
 template <bool FP8>
@@ -135,18 +139,17 @@ __global__ void __launch_bounds__(kScoreThreads, 1)
 score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_constant__ CUtensorMap map_klo,
                     const uint8_t* __restrict__ q, const SegInfo* __restrict__ segs, const float* __restrict__ q_scale,
                     DevParams P, int64_t* __restrict__ seg_offset, int32_t* __restrict__ seg_count,
-                    int32_t* __restrict__ blk_idx, int* __restrict__ work_counter, int* __restrict__ status) {
+                    int32_t* __restrict__ blk_idx, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem;                                    // 2 x 32 KB query tiles
-  uint8_t* sStage = smem + 2 * 32768;                    // kScoreStages x 32 KB pieces (kbar_hi or kbar_lo chunk)
-  float* sS = reinterpret_cast<float*>(sStage + kScoreStages * 32768);  // per candidate: S_J, later E_J
-  float* sM = sS + kMaxBlocks;                                          // per candidate: m_J
-  float* sC = sM + kMaxBlocks;                                          // [2][128] per-row logit multiplier (FP8)
+  uint8_t* sQ = smem;                                    // kScoreQBufs x 32 KB query tiles
+  uint8_t* sStage = smem + kScoreQBufs * 32768;                    // kScoreStages x 32 KB pieces (kbar_hi or kbar_lo chunk)
+  float* sE = reinterpret_cast<float*>(sStage + kScoreStages * 32768);  // per candidate: log2 of its energy
+  float* sC = sE + kMaxBlocks;                                          // [kScoreQBufs][128] per-row multiplier (FP8)
 
-  __shared__ SegInfo info[2];
-  __shared__ int info_valid[2];
-  __shared__ uint64_t info_full[2], info_empty[2], q_full[2], q_empty[2];
+  __shared__ SegInfo info[kScoreInfoSlots];
+  __shared__ int info_valid[kScoreInfoSlots];
+  __shared__ uint64_t info_full[kScoreInfoSlots], info_empty[kScoreInfoSlots], q_full[kScoreQBufs], q_empty[kScoreQBufs];
   __shared__ uint64_t full[kScoreStages], empty[kScoreStages], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
@@ -158,11 +161,15 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
 
   if (tid == 0) {
     abort_flag = 0;
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kScoreInfoSlots; ++i) {
       mbar_init(&info_full[i], 1);
       mbar_init(&info_empty[i], 2 + 256);
+    }
+    for (int i = 0; i < kScoreQBufs; ++i) {
       mbar_init(&q_full[i], 64);
       mbar_init(&q_empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
       mbar_init(&acc_full[i], 1);
       mbar_init(&acc_empty[i], 128);
     }
@@ -182,30 +189,43 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
   const uint32_t tmem = tmem_base_s;
 
   if (warp >= 10) {
-    // ---------------- set-up: next segment (heaviest first), query tile into the free Q buffer ----------------
+    // ---------------- set-up: segment k of this CTA is number blockIdx.x + k * gridDim.x in heaviest-first order
+    // (a static round-robin: no atomic on the critical path).  The loop is software-pipelined: the copies of
+    // tile k+1 are issued before the copies of tile k are waited for, so two query tiles are in flight.
     const int t64 = tid - 320;
-    for (int it = 0;; ++it) {
-      const int slot = it & 1;
-      if (it >= 2) mbar_wait(&info_empty[slot], ((it >> 1) - 1) & 1, ctx, 111);
+    auto seg_of = [&](int k) { return P.nseg - 1 - ((int)blockIdx.x + k * (int)gridDim.x); };
+    auto issue = [&](int k) -> bool {   // publishes tile k's descriptor and starts its query copies
+      const int slot = k % kScoreInfoSlots, qb = k % kScoreQBufs;
+      if (k >= kScoreInfoSlots) mbar_wait(&info_empty[slot], ((k / kScoreInfoSlots) - 1) & 1, ctx, 111);
+      const int sgi = seg_of(k);
+      const bool valid = sgi >= 0;
       if (t64 == 0) {
-        const int w = atomicAdd(work_counter, 1);
-        info_valid[slot] = w < P.nseg;
-        if (w < P.nseg) info[slot] = segs[P.nseg - 1 - w];
+        info_valid[slot] = valid;
+        if (valid) info[slot] = segs[sgi];
       }
       named_bar_sync(2, 64);
-      const bool valid = info_valid[slot] != 0;
       if (t64 == 0) mbar_arrive(&info_full[slot]);
-      if (!valid) break;
+      if (!valid) return false;
       const SegInfo sg = info[slot];
-      if (it >= 2) mbar_wait(&q_empty[slot], ((it >> 1) - 1) & 1, ctx, 112);
-      if constexpr (FP8) load_q_tile_bf16<true, 8>(sQ + slot * 32768, q, sg, P, t64, 64);
-      else load_q_tile_async(sQ + slot * 32768, q, sg, P, t64, 64);
+      // the Q buffer is free once every MMA of the tile that used it kScoreQBufs tiles ago has completed
+      if (k >= kScoreQBufs) mbar_wait(&q_empty[qb], ((k / kScoreQBufs) - 1) & 1, ctx, 112);
       if constexpr (FP8) {
+        load_q_tile_bf16<true, 8>(sQ + qb * 32768, q, sg, P, t64, 64);
         for (int j = t64; j < kTileRows; j += 64)
-          sC[slot * 128 + j] = P.scale_log2 * q_scale[sg.h * P.group + (sg.r0 + j) % P.group];
+          sC[qb * 128 + j] = P.scale_log2 * q_scale[sg.h * P.group + (sg.r0 + j) % P.group];
+      } else {
+        load_q_tile_async(sQ + qb * 32768, q, sg, P, t64, 64, false);
       }
+      cp_async_commit();
+      return true;
+    };
+    bool have = issue(0);
+    for (int k = 0; have; ++k) {
+      const bool next = issue(k + 1);
+      if (next) cp_async_wait_group<1>(); else cp_async_wait_group<0>();
       fence_proxy_async();
-      mbar_arrive(&q_full[slot]);
+      mbar_arrive(&q_full[k % kScoreQBufs]);
+      have = next;
     }
   } else if (warp == 8) {
     // ---------------- producer: kbar pieces (hi, lo of every 128-block chunk) via TMA ----------------
@@ -214,8 +234,8 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       tma_prefetch_desc(&map_klo);
       uint32_t pc = 0;
       for (int it = 0;; ++it) {
-        const int slot = it & 1;
-        mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 121);
+        const int slot = it % kScoreInfoSlots;
+        mbar_wait(&info_full[slot], (it / kScoreInfoSlots) & 1, ctx, 121);
         if (!info_valid[slot]) break;
         const int h = info[slot].h, blk_off = info[slot].blk_off;
         const int nchunks = (info[slot].J_hi + 128) >> 7;
@@ -240,12 +260,12 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       constexpr uint32_t idesc = make_idesc(128, 128, 1, 1, 0, 0);
       uint32_t pc = 0, ac0 = 0, ac1 = 0;
       for (int it = 0;; ++it) {
-        const int slot = it & 1;
-        mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 131);
+        const int slot = it % kScoreInfoSlots, qb = it % kScoreQBufs;
+        mbar_wait(&info_full[slot], (it / kScoreInfoSlots) & 1, ctx, 131);
         if (!info_valid[slot]) break;
         const int nchunks = (info[slot].J_hi + 128) >> 7;
-        mbar_wait(&q_full[slot], (it >> 1) & 1, ctx, 132);
-        const uint32_t q_addr = smem_u32(sQ + slot * 32768);
+        mbar_wait(&q_full[qb], (it / kScoreQBufs) & 1, ctx, 132);
+        const uint32_t q_addr = smem_u32(sQ + qb * 32768);
         for (int c = 0; c < nchunks; ++c) {
           const int a = c & 1;
           uint32_t& ac = a ? ac1 : ac0;
@@ -268,7 +288,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
           }
           umma_commit(&acc_full[a]);
         }
-        umma_commit(&q_empty[slot]);
+        umma_commit(&q_empty[qb]);
         mbar_arrive(&info_empty[slot]);
       }
     }
@@ -280,75 +300,71 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
     const float cs = P.scale_log2;
     uint32_t uc = 0;  // uses of this warpgroup's accumulator
     for (int it = 0;; ++it) {
-      const int slot = it & 1;
-      mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 141);
+      const int slot = it % kScoreInfoSlots, qb = it % kScoreQBufs;
+      mbar_wait(&info_full[slot], (it / kScoreInfoSlots) & 1, ctx, 141);
       if (!info_valid[slot]) break;
       const SegInfo sg = info[slot];
-      const int seg = sg.h_seg();
+      const int seg = sg.seg;
       const int ncand = sg.J_hi + 1;
       const int nchunks = (ncand + 127) >> 7;
+      // per candidate: log2 of its energy, e_J = m_J + log2(S_J)  (Eq. 1-2 / Eq. 20 in the log domain: the
+      // common factor 2^-M of Eq. 20 cancels in the comparison with alpha * max)
+      float lmax = -INFINITY;
       for (int c = wg; c < nchunks; c += 2, ++uc) {
         mbar_wait(&acc_full[wg], uc & 1, ctx, 142);
         tc_fence_after();
         float m, sum;
-        if (sg.nrows == kTileRows) score_chunk<FP8, false>(lane_addr, cs, sC + slot * 128, kTileRows, &acc_empty[wg], m, sum);
-        else score_chunk<FP8, true>(lane_addr, cs, sC + slot * 128, sg.nrows, &acc_empty[wg], m, sum);
+        if (sg.nrows == kTileRows) score_chunk<FP8, false>(lane_addr, cs, sC + qb * 128, kTileRows, &acc_empty[wg], m, sum);
+        else score_chunk<FP8, true>(lane_addr, cs, sC + qb * 128, sg.nrows, &acc_empty[wg], m, sum);
         const int J = c * 128 + key;
         if (J < ncand) {
-          sS[J] = sum;
-          sM[J] = m;
+          const float e = m + log2f(sum);
+          sE[J] = e;
+          lmax = fmaxf(lmax, e);
         }
       }
-      // ---------------- selection: all 256 consumer threads ----------------
-      named_bar_sync(1, 256);
-      float lm = -INFINITY;
-      for (int J = tid; J < ncand; J += 256) lm = fmaxf(lm, sM[J]);
+      // ---------------- selection: all 256 consumer threads, three barriers per tile ----------------
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) lm = fmaxf(lm, __shfl_xor_sync(0xffffffffu, lm, o));
-      if (lane == 0) red[warp] = lm;
-      named_bar_sync(1, 256);
-      float M = red[0];
-#pragma unroll
-      for (int i = 1; i < 8; ++i) M = fmaxf(M, red[i]);
-      named_bar_sync(1, 256);
-      float le = 0.f;
-      for (int J = tid; J < ncand; J += 256) {
-        const float e = sS[J] * exp2f(sM[J] - M);
-        sS[J] = e;
-        le = fmaxf(le, e);
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) le = fmaxf(le, __shfl_xor_sync(0xffffffffu, le, o));
-      if (lane == 0) red[warp] = le;
-      named_bar_sync(1, 256);
+      for (int o = 16; o > 0; o >>= 1) lmax = fmaxf(lmax, __shfl_xor_sync(0xffffffffu, lmax, o));
+      if (lane == 0) red[warp] = lmax;
+      named_bar_sync(1, 256);            // energies and per-warp maxima are visible
       float maxE = red[0];
 #pragma unroll
       for (int i = 1; i < 8; ++i) maxE = fmaxf(maxE, red[i]);
-      const float thr = P.alpha * maxE;
+      // J selected  <=>  E_J >= alpha max E  <=>  e_J >= log2(alpha) + max e   (alpha <= 0 selects everything)
+      const float thr = P.alpha > 0.f ? maxE + log2f(P.alpha) : -INFINITY;
       const int win_lo = sg.J_lo - P.window_blocks;
-      int base = 0;
-      for (int J0 = 0; J0 < ncand; J0 += 256) {
-        const int J = J0 + tid;
-        const bool keep = J < ncand && (sS[J] >= thr || J < P.sink_blocks || J >= win_lo);
-        const unsigned bal = __ballot_sync(0xffffffffu, keep);
-        if (lane == 0) wsum[warp] = __popc(bal);
-        named_bar_sync(1, 256);
-        int before = 0, total = 0;
+      // warp w owns candidates [w * per, (w + 1) * per), per a multiple of 32: count, exchange, write in order
+      const int per = (((ncand + 7) >> 3) + 31) & ~31;
+      const int beg = warp * per, end = min(beg + per, ncand);
+      int mine = 0;
+      for (int J0 = beg; J0 < end; J0 += 32) {
+        const int J = J0 + lane;
+        const bool keep = J < end && (sE[J] >= thr || J < P.sink_blocks || J >= win_lo);
+        mine += __popc(__ballot_sync(0xffffffffu, keep));
+      }
+      if (lane == 0) wsum[warp] = mine;
+      named_bar_sync(1, 256);
+      int pos = 0, total = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int v = wsum[i];
-          before += (i < warp) ? v : 0;
-          total += v;
-        }
-        if (keep) blk_idx[sg.off + base + before + __popc(bal & ((1u << lane) - 1u))] = J;
-        base += total;
-        named_bar_sync(1, 256);
+      for (int i = 0; i < 8; ++i) {
+        const int v = wsum[i];
+        pos += (i < warp) ? v : 0;
+        total += v;
+      }
+      for (int J0 = beg; J0 < end; J0 += 32) {
+        const int J = J0 + lane;
+        const bool keep = J < end && (sE[J] >= thr || J < P.sink_blocks || J >= win_lo);
+        const unsigned bal = __ballot_sync(0xffffffffu, keep);
+        if (keep) blk_idx[sg.off + pos + __popc(bal & ((1u << lane) - 1u))] = J;
+        pos += __popc(bal);
       }
       if (tid == 0) {
-        seg_count[seg] = base;
+        seg_count[seg] = total;
         seg_offset[seg] = sg.off;
         if (seg == P.nseg - 1) seg_offset[P.nseg] = sg.off + ncand;
       }
+      named_bar_sync(1, 256);            // sE, red and wsum are reused by the next tile
       mbar_arrive(&info_empty[slot]);
     }
   }
