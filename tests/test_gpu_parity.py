@@ -116,6 +116,64 @@ def test_config5_relative_batch_with_prefixes():
     assert len(spec.seqs) == 16 and any(pre > 0 for _, pre in spec.seqs)
 
 
+def _sampled_segments(wl, heads, tiles_per_head, seed):
+    """First, last and random tiles of the given KV heads of sequence 0 (full-size workloads)."""
+    rng = np.random.default_rng(seed)
+    by_head = {}
+    for s in wl.segs:
+        if s.b == 0:
+            by_head.setdefault(s.h, []).append(s.seg)
+    ids = set()
+    for h in heads:
+        segs = by_head[h]
+        n = len(segs)
+        pick = {0, 1, n // 2, n - 2, n - 1} | set(rng.integers(0, n, tiles_per_head).tolist())
+        ids |= {segs[i] for i in pick}
+    return sorted(ids)
+
+
+def test_config3_full_size_in_the_bench_configuration_sampled():
+    """131072 tokens, the launch configuration bench.py times (alpha near 95 % sparsity): lists and
+    attention of sampled segments against the oracle, plus properties that hold at any size."""
+    spec = inputs.config_spec(3)
+    spec.alpha = 4.6e-3
+    case, dc, wl = make(spec)
+    dc.select(); dc.status()
+    cnt = dc.seg_count.cpu().numpy()
+    off = dc.seg_offset.cpu().numpy()
+    assert off[-1] == dc.plan.idx_capacity == 8 * 2099200
+    sparsity = 1.0 - cnt.sum() / dc.plan.idx_capacity
+    assert 0.93 < sparsity < 0.97
+    # any-size properties: counts within candidates, forced blocks present, lists ascending
+    idx = dc.blk_idx.cpu().numpy()
+    for s in wl.segs[:: 97]:
+        l = idx[off[s.seg]: off[s.seg] + cnt[s.seg]]
+        assert 1 <= len(l) <= s.J_hi + 1 and np.all(np.diff(l) > 0) and l[-1] == s.J_hi
+        assert set(range(s.J_lo, s.J_hi + 1)) <= set(l.tolist())
+    ids = _sampled_segments(wl, heads=(0, 5), tiles_per_head=3, seed=3)
+    check_lists(dc, wl, ids)
+    lists = {i: idx[off[i]: off[i] + cnt[i]].copy() for i in ids}
+    dc.sparse(); dc.status()
+    check_attention(dc, wl, lists, ids)
+    assert torch.isfinite(dc.out.float()).all() and torch.isfinite(dc.lse).all()
+    dc.dense(); dc.status()
+    check_attention(dc, wl, None, ids[:3] + ids[-2:], dense=True)
+
+
+def test_config5_full_size_sampled():
+    """The continuous batch at full size (16 sequences, ~256K KV tokens, 16-token pages, prefixes)."""
+    spec = inputs.config_spec(5)
+    case, dc, wl = make(spec)
+    dc.select(); dc.status()
+    rng = np.random.default_rng(5)
+    ids = sorted(set(rng.integers(0, len(wl.segs), 24).tolist()) | {0, len(wl.segs) - 1})
+    check_lists(dc, wl, ids)
+    lists_all = dc.lists_host()
+    dc.sparse(); dc.status()
+    check_attention(dc, wl, {i: lists_all[i] for i in ids}, ids)
+    assert torch.isfinite(dc.out.float()).all()
+
+
 # ------------------------------------------------------------------------------------------------------
 # edge cases
 # ------------------------------------------------------------------------------------------------------
