@@ -34,7 +34,7 @@ struct fp2_plan {
   SegInfo* d_segs;
   int32_t* d_blk_off;
   // workspace layout (byte offsets)
-  int64_t ws_status, ws_counter, ws_khi, ws_klo, ws_vbar, ws_order, ws_hist, ws_bytes;
+  int64_t ws_status, ws_counter, ws_khi, ws_klo, ws_vbar, ws_kf16, ws_order, ws_hist, ws_bytes;
   EncodeTiledFn encode;
   int32_t last_launches;
   bool attrs_set;
@@ -173,6 +173,7 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
   pl->ws_khi = o;  o += pooled;
   pl->ws_klo = o;  o += pooled;
   pl->ws_vbar = o; o += pooled;
+  pl->ws_kf16 = o; o += (p->dtype == FP2_FP8_E4M3) ? pooled : 0;
   pl->ws_order = o; o += align_up(4 * (pl->nseg > 0 ? pl->nseg : 1), 1024);
   pl->ws_hist = o;  o += align_up(4 * ((int64_t)p->num_kv_heads * kCountBuckets + 1), 1024);
   pl->ws_bytes = o;
@@ -242,7 +243,9 @@ static fp2_status set_attrs(fp2_plan* pl) {
       cudaFuncSetAttribute(score_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kScoreSmemBytes) != cudaSuccess ||
       cudaFuncSetAttribute(sparse_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           kAttnSmemBytes) != cudaSuccess)
+                           AttnCfg<false>::kSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(sparse_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           AttnCfg<true>::kSmemBytes) != cudaSuccess)
     return FP2_ERR_CUDA;
   pl->attrs_set = true;
   return FP2_OK;
@@ -270,12 +273,13 @@ static fp2_status launch_pool(fp2_plan* pl, const void* k, const void* v, const 
   __nv_bfloat16* khi = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_khi);
   __nv_bfloat16* klo = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_klo);
   __nv_bfloat16* vb = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_vbar);
+  __half* kf16 = reinterpret_cast<__half*>(ws + pl->ws_kf16);
   if (pl->dev.fp8)
     pool_kv_kernel<true><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, lk, pl->d_blk_off, ks, vs,
-                                               pl->dev, khi, klo, vb);
+                                               pl->dev, khi, klo, vb, kf16);
   else
     pool_kv_kernel<false><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, lk, pl->d_blk_off, ks, vs,
-                                                pl->dev, khi, klo, vb);
+                                                pl->dev, khi, klo, vb, kf16);
   pl->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
@@ -337,7 +341,6 @@ static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, cons
   fp2_status s = check_common(pl, q, k, v, pt, cu, lk, qs, ks, vs, workspace);
   if (s != FP2_OK) return s;
   if (!out || !aligned(out, 16)) return FP2_ERR_INVALID_ARG;
-  if (pl->dev.fp8) return FP2_ERR_UNSUPPORTED;  // FP8 attention kernel not built yet
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   pl->last_launches = 0;
@@ -349,7 +352,7 @@ static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, cons
   CUtensorMap mk, mv, mkb, mvb;
   if (!make_map(pl, &mk, k, slots, pl->prm.num_kv_heads, pl->prm.page_size, fp8) ||
       !make_map(pl, &mv, v, slots, pl->prm.num_kv_heads, pl->prm.page_size, fp8) ||
-      !make_map(pl, &mkb, ws + pl->ws_khi, pl->nblk_tot, pl->prm.num_kv_heads, 128, false) ||
+      !make_map(pl, &mkb, ws + (fp8 ? pl->ws_kf16 : pl->ws_khi), pl->nblk_tot, pl->prm.num_kv_heads, 128, false) ||
       !make_map(pl, &mvb, ws + pl->ws_vbar, pl->nblk_tot, pl->prm.num_kv_heads, 128, false))
     return FP2_ERR_CUDA;
   AttnArgs a;
@@ -365,7 +368,12 @@ static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, cons
   a.work_counter = reinterpret_cast<int*>(ws + pl->ws_counter);
   a.status = reinterpret_cast<int*>(ws + pl->ws_status);
   const unsigned grid = (unsigned)(pl->nseg < pl->num_sms ? pl->nseg : pl->num_sms);
-  sparse_attn_kernel<false><<<grid, kAttnThreads, kAttnSmemBytes, st>>>(mk, mv, mkb, mvb, a, pl->dev);
+  if (fp8)
+    sparse_attn_kernel<true><<<grid, AttnCfg<true>::kThreads, AttnCfg<true>::kSmemBytes, st>>>(mk, mv, mkb, mvb, a,
+                                                                                              pl->dev);
+  else
+    sparse_attn_kernel<false><<<grid, AttnCfg<false>::kThreads, AttnCfg<false>::kSmemBytes, st>>>(mk, mv, mkb, mvb,
+                                                                                                 a, pl->dev);
   pl->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
@@ -464,7 +472,8 @@ extern "C" fp2_status fp2_dense_prefill_static(fp2_plan* pl, const void* q, cons
   a.status = reinterpret_cast<int*>(sw);
   const unsigned grid = (unsigned)(pl->nseg < pl->num_sms ? pl->nseg : pl->num_sms);
   // the dense path stages no pooled chunks: the two pooled-mean maps are never dereferenced
-  sparse_attn_kernel<false><<<grid, kAttnThreads, kAttnSmemBytes, st>>>(mk, mv, mk, mv, a, pl->dev);
+  sparse_attn_kernel<false><<<grid, AttnCfg<false>::kThreads, AttnCfg<false>::kSmemBytes, st>>>(mk, mv, mk, mv, a,
+                                                                                               pl->dev);
   pl->last_launches = 4;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }

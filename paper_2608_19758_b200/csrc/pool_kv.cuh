@@ -6,8 +6,12 @@
 //   kbar_hi = bf16(mean k), kbar_lo = bf16(mean k - kbar_hi)   (hi + lo carries ~16 mantissa bits for the scorer)
 //   vbar    = bf16(mean v)
 // kbar_hi and vbar double as the operands of the correction chunks in the attention kernel.
+// FP8 inputs: kbar_hi / kbar_lo hold the de-scaled mean (mean of raw values x k_scale); the attention kernel
+// runs its MMAs on F16 copies of the raw e4m3 values, so for its correction chunks this kernel also writes
+// kbar_f16 = f16(de-scaled mean k) and stores vbar as f16(mean of RAW v) -- v_scale is applied to the output.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_fp8.h>
 #include "common.cuh"
 
@@ -47,7 +51,8 @@ __global__ void __launch_bounds__(256) pool_kv_kernel(const uint8_t* __restrict_
                                                       const float* __restrict__ v_scale, DevParams P,
                                                       __nv_bfloat16* __restrict__ kbar_hi,
                                                       __nv_bfloat16* __restrict__ kbar_lo,
-                                                      __nv_bfloat16* __restrict__ vbar) {
+                                                      __nv_bfloat16* __restrict__ vbar,
+                                                      __half* __restrict__ kbar_f16) {
   constexpr int ROW_BYTES = FP8 ? 128 : 256;
   constexpr int CHUNKS = ROW_BYTES / 16;       // 16-byte chunks per token row
   constexpr int EPC = FP8 ? 16 : 8;            // elements per chunk
@@ -104,14 +109,16 @@ __global__ void __launch_bounds__(256) pool_kv_kernel(const uint8_t* __restrict_
 #pragma unroll
   for (int r = 0; r < ROWS_PER_PASS; ++r) s += red[which][r][c];
   float mean = s / (float)ntok;
-  if constexpr (FP8) mean *= (which == 0 ? k_scale[h] : v_scale[h]);
+  if constexpr (FP8) mean *= (which == 0 ? k_scale[h] : 1.0f);
   const size_t o = ((size_t)gblk * P.num_kv_heads + h) * kHeadDim + c;
   const __nv_bfloat16 hi16 = __float2bfloat16_rn(mean);
   if (which == 0) {
     kbar_hi[o] = hi16;
     kbar_lo[o] = __float2bfloat16_rn(mean - __bfloat162float(hi16));
+    if constexpr (FP8) kbar_f16[o] = __float2half_rn(mean);
   } else {
-    vbar[o] = hi16;
+    if constexpr (FP8) reinterpret_cast<__half*>(vbar)[o] = __float2half_rn(mean);
+    else vbar[o] = hi16;
   }
 }
 

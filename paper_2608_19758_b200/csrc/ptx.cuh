@@ -242,6 +242,18 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return d;
 }
 
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+// two e4m3 bytes (low 16 bits of x) -> two f16 (exact)
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t x) {
+  uint32_t d;
+  asm("{\n .reg .b16 t;\n cvt.u16.u32 t, %1;\n cvt.rn.f16x2.e4m3x2 %0, t;\n}" : "=r"(d) : "r"(x));
+  return d;
+}
+
 // Byte offset of element column-chunk `chunk16` (16-byte units within a 128-byte row) of row `row` inside a
 // 128-byte-swizzled tile whose base is 1024-byte aligned.
 __device__ __forceinline__ uint32_t sw128_offset(int row, int chunk16) {

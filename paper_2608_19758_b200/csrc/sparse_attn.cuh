@@ -16,6 +16,7 @@
 //   warp 8     TMA producer: K / V pages through the page table into two rings (Eq. 22)
 //   warp 9     UMMA issuer: S = Q K^T (SS), O += P V (P read from TMEM, V MN-major from shared memory)
 //   warps 10-11 tile set-up: fetch the next unit, validate its list, build the correction masks, stage Q
+//   warps 12-15 (FP8 inputs only) widen raw e4m3 K / V tiles to F16 into the K / V rings
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512).  P (BF16 pairs) has its own
 // columns, so S = Q K^T of iteration i+2 may start as soon as the softmax of iteration i has read S -- it does
@@ -30,11 +31,23 @@
 
 namespace fp2 {
 
-constexpr int kAttnThreads = 384;
-constexpr int kNK = 3;  // K ring stages (32 KB each)
-constexpr int kNV = 2;  // V ring stages
-constexpr int kTileBytes = 32768;
-constexpr int kAttnSmemBytes = 1024 + kTileBytes * (1 + kNK + kNV) + 3072;
+constexpr int kTileBytes = 32768;   // one 128 x 128 tile of 16-bit elements
+constexpr int kRawBytes = 16384;    // one 128 x 128 tile of FP8 elements as TMA delivers it
+
+// FP8 inputs (Eq. 15) run through the same 16-bit pipeline: the producer lands raw e4m3 K / V tiles in a small
+// ring, a fourth warpgroup widens them to F16 (exact) into the K / V rings, and both GEMMs run as kind::f16
+// with F16 operands (Q widened when staged, P packed as F16).  The per-head scales never touch the operands:
+// q_scale * k_scale multiplies the logits of a row, v_scale multiplies the output.  A single e4m3 probability
+// tile, the other way to feed FP8 V to the tensor core, costs ~0.06 max-abs output error by itself.
+template <bool FP8>
+struct AttnCfg {
+  static constexpr int kThreads = FP8 ? 512 : 384;
+  static constexpr int kNK = FP8 ? 2 : 3;   // K ring stages (32 KB each)
+  static constexpr int kNV = 2;             // V ring stages
+  static constexpr int kNRaw = FP8 ? 3 : 0; // raw FP8 tile ring (16 KB each), K and V tiles alternate
+  static constexpr int kSmemBytes = 1024 + kTileBytes * (1 + kNK + kNV) + kNRaw * kRawBytes + 3072;
+  static constexpr int kFmt = FP8 ? 0 : 1;  // UMMA kind::f16 operand format: 0 = F16, 1 = BF16
+};
 
 struct TileInfo {
   SegInfo sg;
@@ -101,6 +114,7 @@ __device__ __forceinline__ float half_row_max(uint32_t s_addr) {
 
 // p = 2^(s * cs + neg_m) for this thread's 64 columns, written as BF16 pairs to 32 columns at p_addr.
 // The second TMEM load is in flight while the first half is exponentiated.  Returns the row's partial sum.
+template <bool F16>
 __device__ __forceinline__ float half_row_exp(uint32_t s_addr, uint32_t p_addr, float cs, float neg_m) {
   float sum4[4] = {0.f, 0.f, 0.f, 0.f};
   uint32_t buf[2][32];
@@ -115,7 +129,7 @@ __device__ __forceinline__ float half_row_exp(uint32_t s_addr, uint32_t p_addr, 
       const float p0 = ex2(fmaf(__uint_as_float(buf[k][2 * j]), cs, neg_m));
       const float p1 = ex2(fmaf(__uint_as_float(buf[k][2 * j + 1]), cs, neg_m));
       sum4[j & 3] += p0 + p1;
-      pk[j] = pack_bf16x2(p0, p1);
+      pk[j] = F16 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1);
     }
     if (k == 0) tmem_wait_ld();
     tmem_st16(p_addr + k * 16, pk);
@@ -123,24 +137,80 @@ __device__ __forceinline__ float half_row_exp(uint32_t s_addr, uint32_t p_addr, 
   return (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
 }
 
+// FP8 query tile -> shared memory as F16 (exact), same K-major swizzled layout as the BF16 tile.
+__device__ __forceinline__ void load_q_tile_f16(uint8_t* sQ, const uint8_t* __restrict__ q, const SegInfo& sg,
+                                                const DevParams& P, int t, int nthr) {
+  const int g = P.group;
+  constexpr int BATCH = 8;
+  for (int i0 = t; i0 < kTileRows * 16; i0 += nthr * BATCH) {
+    uint2 v[BATCH];
+#pragma unroll
+    for (int u = 0; u < BATCH; ++u) {
+      const int i = i0 + u * nthr;
+      const int row = i >> 4, ch = i & 15;   // 16 chunks of 8 elements per row
+      v[u] = make_uint2(0, 0);
+      if (i < kTileRows * 16 && row < sg.nrows) {
+        const int r = sg.r0 + row;
+        const size_t tok = (size_t)sg.q_tok0 + r / g;
+        const size_t head = (size_t)sg.h * g + r % g;
+        v[u] = __ldg(reinterpret_cast<const uint2*>(q + (tok * P.num_q_heads + head) * kHeadDim + ch * 8));
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < BATCH; ++u) {
+      const int i = i0 + u * nthr;
+      const int row = i >> 4, ch = i & 15;
+      if (i < kTileRows * 16) {
+        const uint4 o = make_uint4(e4m3x2_to_f16x2(v[u].x), e4m3x2_to_f16x2(v[u].x >> 16),
+                                   e4m3x2_to_f16x2(v[u].y), e4m3x2_to_f16x2(v[u].y >> 16));
+        *reinterpret_cast<uint4*>(sQ + (ch >> 3) * 16384 + sw128_offset(row, ch & 7)) = o;
+      }
+    }
+  }
+}
+
+// One raw FP8 tile (128 rows x 128 bytes, 128-byte swizzle as TMA wrote it) -> one F16 tile in the two-halves
+// layout of the K / V rings.  128 threads; eight consecutive threads take one row, so every quarter-warp reads
+// one whole 128-byte row (conflict-free).  Element order inside a row is preserved, so the same routine
+// serves K (K-major operand) and V (MN-major operand).
+__device__ __forceinline__ void widen_tile_f16(const uint8_t* raw, uint8_t* dst, int t) {
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const int i = t + 128 * k;
+    const int row = i >> 3, c = i & 7;        // c: 16-byte chunk = 16 elements d = 16c .. 16c+15
+    const uint4 v = *reinterpret_cast<const uint4*>(raw + sw128_offset(row, c));
+    const uint4 lo = make_uint4(e4m3x2_to_f16x2(v.x), e4m3x2_to_f16x2(v.x >> 16), e4m3x2_to_f16x2(v.y),
+                                e4m3x2_to_f16x2(v.y >> 16));
+    const uint4 hi = make_uint4(e4m3x2_to_f16x2(v.z), e4m3x2_to_f16x2(v.z >> 16), e4m3x2_to_f16x2(v.w),
+                                e4m3x2_to_f16x2(v.w >> 16));
+    uint8_t* half = dst + (c >> 2) * 16384;   // d < 64 -> first half
+    const int oc = (c & 3) * 2;               // chunk index inside the half (8 f16 per 16 bytes)
+    *reinterpret_cast<uint4*>(half + sw128_offset(row, oc)) = lo;
+    *reinterpret_cast<uint4*>(half + sw128_offset(row, oc + 1)) = hi;
+  }
+}
+
 template <bool FP8>
-__global__ void __launch_bounds__(kAttnThreads, 1)
+__global__ void __launch_bounds__(AttnCfg<FP8>::kThreads, 1)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                    const __grid_constant__ CUtensorMap map_kbar, const __grid_constant__ CUtensorMap map_vbar,
                    AttnArgs A, DevParams P) {
-  static_assert(!FP8, "FP8 path is built separately");
+  constexpr int kNK = AttnCfg<FP8>::kNK, kNV = AttnCfg<FP8>::kNV, kNRaw = AttnCfg<FP8>::kNRaw;
+  constexpr int kAttnThreads = AttnCfg<FP8>::kThreads;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = smem;
   uint8_t* sK = smem + kTileBytes;
   uint8_t* sV = sK + kNK * kTileBytes;
-  float* sX = reinterpret_cast<float*>(sV + kNV * kTileBytes);   // [2 parity][2 wg][128] row-max / row-sum exchange
+  uint8_t* sRaw = sV + kNV * kTileBytes;                          // FP8 only: raw tile ring
+  float* sX = reinterpret_cast<float*>(sRaw + kNRaw * kRawBytes);  // [2 parity][2 wg][128] row-max / row-sum exchange
 
   __shared__ TileInfo info[2];
   __shared__ uint32_t sel_bits[2][kMaxBlocks / 32];
   __shared__ uint64_t info_full[2], info_empty[2], q_full, q_empty, tile_done;
   __shared__ uint64_t k_full[kNK], k_empty[kNK], v_full[kNV], v_empty[kNV];
   __shared__ uint64_t s_full[2], p_ready[2], o_done;
+  __shared__ uint64_t raw_full[kNRaw > 0 ? kNRaw : 1], raw_empty[kNRaw > 0 ? kNRaw : 1];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
 
@@ -151,7 +221,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     abort_flag = 0;
     for (int i = 0; i < 2; ++i) {
       mbar_init(&info_full[i], 1);
-      mbar_init(&info_empty[i], 2 + 256);
+      mbar_init(&info_empty[i], 2 + 256 + (FP8 ? 1 : 0));
       mbar_init(&s_full[i], 1);
       mbar_init(&p_ready[i], 256);
     }
@@ -161,11 +231,12 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     mbar_init(&o_done, 1);
     for (int i = 0; i < kNK; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
     for (int i = 0; i < kNV; ++i) { mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); }
+    for (int i = 0; i < kNRaw; ++i) { mbar_init(&raw_full[i], 1); mbar_init(&raw_empty[i], 1); }
     fence_barrier_init();
   }
   // K / V rings start zeroed: rows of pages past the end of a sequence are never loaded, and whatever sits
   // there is multiplied by probabilities that are exactly zero, so it must be finite.
-  for (int i = tid; i < (kNK + kNV) * kTileBytes / 16; i += kAttnThreads)
+  for (int i = tid; i < ((kNK + kNV) * kTileBytes + kNRaw * kRawBytes) / 16; i += kAttnThreads)
     reinterpret_cast<uint4*>(sK)[i] = make_uint4(0, 0, 0, 0);
   if (warp == 9) {
     tmem_alloc(&tmem_base_s, 512);
@@ -178,7 +249,43 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
   const uint32_t tmem = tmem_base_s;
   const int g = P.group;
 
-  if (warp >= 10) {
+  if (FP8 && warp >= 12) {
+    // =============================== FP8 -> F16 widening warpgroup ===============================
+    setmaxnreg_dec<56>();
+    if constexpr (FP8) {
+      const int t128 = tid - 384;
+      uint32_t kc = 0, vc = 0, rc = 0;
+      for (int it = 0;; ++it) {
+        const int slot = it & 1;
+        mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 601);
+        const TileInfo& ti = info[slot];
+        if (!ti.valid) break;
+        const int T = ti.T, n_it = T + ti.nchunk;
+        for (int i = 0; i < n_it; ++i, ++kc, ++vc) {
+          if (i >= T) continue;   // correction chunks arrive as F16 straight into the K / V rings
+#pragma unroll
+          for (int kv = 0; kv < 2; ++kv, ++rc) {
+            const int rs = rc % kNRaw;
+            const int ds = kv ? (int)(vc % kNV) : (int)(kc % kNK);
+            const uint32_t dc = kv ? vc : kc;
+            const int dn = kv ? kNV : kNK;
+            uint64_t* d_empty = kv ? &v_empty[ds] : &k_empty[ds];
+            uint64_t* d_full = kv ? &v_full[ds] : &k_full[ds];
+            if (dc >= (uint32_t)dn) mbar_wait(d_empty, ((dc / dn) - 1) & 1, ctx, 602);
+            mbar_wait(&raw_full[rs], (rc / kNRaw) & 1, ctx, 603);
+            widen_tile_f16(sRaw + rs * kRawBytes, (kv ? sV : sK) + ds * kTileBytes, t128);
+            fence_proxy_async();
+            named_bar_sync(3, 128);
+            if (t128 == 0) {
+              mbar_arrive(&raw_empty[rs]);
+              mbar_arrive(d_full);
+            }
+          }
+        }
+        if (t128 == 0) mbar_arrive(&info_empty[slot]);
+      }
+    }
+  } else if (warp >= 10) {
     // =============================== tile set-up + Q staging ===============================
     setmaxnreg_dec<56>();
     const int t64 = tid - 320;
@@ -249,7 +356,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       if (!valid) break;
       // Q tile: wait until every S = Q K^T of the previous unit has completed, then overwrite
       if (it >= 1) mbar_wait(&q_empty, (it - 1) & 1, ctx, 202);
-      load_q_tile_async(sQ, A.q, ti.sg, P, t64, 64);
+      if constexpr (FP8) load_q_tile_f16(sQ, A.q, ti.sg, P, t64, 64);
+      else load_q_tile_async(sQ, A.q, ti.sg, P, t64, 64);
       fence_proxy_async();
       mbar_arrive(&q_full);
     }
@@ -262,7 +370,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       tma_prefetch_desc(&map_kbar);
       tma_prefetch_desc(&map_vbar);
     }
-    uint32_t kc = 0, vc = 0;
+    uint32_t kc = 0, vc = 0, rc = 0;
+    (void)rc;
     const int ppb = P.pages_per_block, psz = P.page_size;
     for (int it = 0;; ++it) {
       const int slot = it & 1;
@@ -292,6 +401,23 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
             }
           }
           const int nvalid = __popc(__ballot_sync(0xffffffffu, pid >= 0));
+          if constexpr (FP8) {
+            // raw e4m3 tiles (128 bytes per token row) into the raw ring; the widening warpgroup fills the K / V rings
+            const uint32_t rbytes = (uint32_t)nvalid * psz * 128u;
+#pragma unroll
+            for (int kv = 0; kv < 2; ++kv, ++rc) {
+              const int rs = rc % kNRaw;
+              if (rc >= (uint32_t)kNRaw) mbar_wait(&raw_empty[rs], ((rc / kNRaw) - 1) & 1, ctx, 306);
+              if (lane == 0) mbar_arrive_expect_tx(&raw_full[rs], rbytes);
+              __syncwarp();
+              if (pid >= 0)
+                tma_load_3d(sRaw + rs * kRawBytes + lane * psz * 128, kv ? &map_v : &map_k, &raw_full[rs], 0, sg.h,
+                            pid * psz);
+            }
+            ++kc;
+            ++vc;
+            continue;
+          }
           const uint32_t bytes = (uint32_t)nvalid * psz * 256u;
           if (kc >= kNK) mbar_wait(&k_empty[ks], ((kc / kNK) - 1) & 1, ctx, 302);
           if (lane == 0) mbar_arrive_expect_tx(&k_full[ks], bytes);
@@ -332,8 +458,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     // =============================== UMMA issuer ===============================
     setmaxnreg_dec<56>();
     if (lane == 0) {
-      constexpr uint32_t idesc_qk = make_idesc(128, 128, 1, 1, 0, 0);
-      constexpr uint32_t idesc_pv = make_idesc(128, 128, 1, 1, 0, 1);
+      constexpr int kFmt = AttnCfg<FP8>::kFmt;
+      constexpr uint32_t idesc_qk = make_idesc(128, 128, kFmt, kFmt, 0, 0);
+      constexpr uint32_t idesc_pv = make_idesc(128, 128, kFmt, kFmt, 0, 1);
       const uint32_t q_addr = smem_u32(sQ);
       uint32_t kc = 0, vc = 0, pc0 = 0, pc1 = 0;
       auto issue_pv = [&](int j) {
@@ -388,14 +515,14 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     }
   } else {
     // =============================== softmax warpgroups + epilogue ===============================
-    setmaxnreg_inc<224>();
+    // register budget: 384 threads: 128 x 56 + 256 x 224 = 64512; 512 threads (FP8): 256 x 56 + 256 x 200 = 65536
+    setmaxnreg_inc<FP8 ? 200 : 224>();
     const int wg = warp >> 2;
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t o_addr = lane_base + 256 + wg * 64;   // this thread's 64 columns of O
     uint32_t sc0 = 0, sc1 = 0;   // completed uses of S0 / S1 (phases of s_full)
     uint32_t pv_base = 0;        // UMMA groups O += P V issued before this tile (phase of o_done)
-    const float cs = P.scale_log2;
     for (int it = 0;; ++it) {
       const int slot = it & 1;
       mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 501);
@@ -406,6 +533,15 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       const int32_t* list = A.blk_idx + sg.off;
       const int r = sg.r0 + row;
       const int pos = sg.pre + r / g;
+      // logit multipliers in log2 units.  FP8 (Eq. 15): the MMAs see raw e4m3 values, so exact blocks carry
+      // q_scale * k_scale and pooled chunks (kbar is stored de-scaled) carry q_scale only.
+      float cs_exact = P.scale_log2, cs_chunk = P.scale_log2, out_scale = 1.0f;
+      if constexpr (FP8) {
+        const float qs = A.q_scale[sg.h * g + r % g];
+        cs_chunk *= qs;
+        cs_exact *= qs * A.k_scale[sg.h];
+        out_scale = A.v_scale[sg.h];
+      }
       float m = -INFINITY, l = 0.f;
       // block id of the next exact iteration, fetched one iteration ahead
       int J_next = (!ti.dense && T > 0) ? list[T - 1] : 0;
@@ -417,7 +553,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         bool need_mask = false;
         int tok_lim = 1 << 30;     // exact block: columns j with j <= tok_lim are visible
         uint32_t cm_lo = 0xffffffffu, cm_hi = 0xffffffffu;
-        float shift = 0.f;
+        float shift = 0.f, cs = cs_exact;
         if (i < T) {
           int J = ti.dense ? sg.J_hi - i : J_next;
           if (!ti.dense && i + 1 < T) J_next = list[T - 2 - i];
@@ -429,6 +565,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           cm_lo = ti.todo[c][2 * wg];
           cm_hi = ti.todo[c][2 * wg + 1];
           shift = 7.0f;  // log2(128): one pooled row stands for a full block (Eq. 6)
+          cs = cs_chunk;
           need_mask = true;
         }
         if (a) { mbar_wait(&s_full[1], sc1 & 1, ctx, 502); ++sc1; }
@@ -467,7 +604,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         }
         // a row with nothing visible so far has m = -inf and only -inf logits: exponent against 0 -> zeros
         const float neg_m = (m == -INFINITY) ? shift : shift - m;
-        l += half_row_exp(s_addr, p_addr, cs, neg_m);
+        l += half_row_exp<FP8>(s_addr, p_addr, cs, neg_m);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&p_ready[a]);
@@ -480,7 +617,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       xch[wg * 128 + row] = l;
       named_bar_sync(1, 256);
       const float L = l + xch[(wg ^ 1) * 128 + row];
-      const float inv = L > 0.f ? 1.0f / L : 0.f;
+      const float inv = L > 0.f ? out_scale / L : 0.f;
       const bool have_o = n_it >= 1;
       const bool row_ok = row < sg.nrows;
       const size_t tok = (size_t)sg.q_tok0 + r / g;

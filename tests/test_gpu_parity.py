@@ -175,6 +175,54 @@ def test_config5_full_size_sampled():
 
 
 # ------------------------------------------------------------------------------------------------------
+# FP8 e4m3 inputs with per-head scales (Eq. 15); oracle on the de-quantised values
+# ------------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("g,hkv,p,seqs", [
+    (7, 2, 64, [(2300, 0)]),
+    (4, 2, 16, [(1500, 300), (700, 0), (129, 128)]),
+    (1, 2, 32, [(900, 100)]),
+])
+def test_fp8_small(g, hkv, p, seqs):
+    spec = inputs.small_spec(seqs=seqs, num_q_heads=g * hkv, num_kv_heads=hkv, page_size=p, dtype="fp8",
+                             config_id=40 + g)
+    spec.alpha = 0.2
+    full_pipeline(spec)
+
+
+def test_fp8_without_sink_and_heavy_pruning():
+    spec = inputs.small_spec(seqs=[(4096, 0)], num_q_heads=8, num_kv_heads=2, page_size=64, dtype="fp8",
+                             config_id=48, sink=False, sink_tokens=0, window_tokens=128)
+    spec.alpha = 0.5
+    case, dc, wl = full_pipeline(spec, dense=False)
+    assert int(dc.seg_count.sum()) < dc.plan.idx_capacity / 2
+
+
+def test_config4_relative_at_16k():
+    spec = inputs.config_spec(4, scale_down=8)
+    full_pipeline(spec)
+
+
+def test_config4_full_size_sampled():
+    """FP8, 131072 tokens, Hq=28 / Hkv=4 (g = 7: tiles straddle positions), sampled segments."""
+    spec = inputs.config_spec(4)
+    spec.alpha = 4.6e-3
+    case, dc, wl = make(spec)
+    dc.select(); dc.status()
+    ids = _sampled_segments(wl, heads=(1, 3), tiles_per_head=3, seed=4)
+    check_lists(dc, wl, ids)
+    lists_all = dc.lists_host()
+    dc.sparse(); dc.status()
+    check_attention(dc, wl, {i: lists_all[i] for i in ids}, ids, dtype="fp8")
+    assert torch.isfinite(dc.out.float()).all()
+
+
+def test_config5_fp8_relative():
+    spec = inputs.config_spec(5, dtype="fp8", scale_down=8)
+    full_pipeline(spec)
+
+
+# ------------------------------------------------------------------------------------------------------
 # edge cases
 # ------------------------------------------------------------------------------------------------------
 
