@@ -34,7 +34,7 @@ struct fp2_plan {
   SegInfo* d_segs;
   int32_t* d_blk_off;
   // workspace layout (byte offsets)
-  int64_t ws_status, ws_counter, ws_khi, ws_klo, ws_vbar, ws_kf16, ws_order, ws_hist, ws_bytes;
+  int64_t ws_status, ws_counter, ws_khi, ws_klo, ws_vbar, ws_order, ws_hist, ws_bytes;
   EncodeTiledFn encode;
   int32_t last_launches;
   bool attrs_set;
@@ -173,7 +173,6 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
   pl->ws_khi = o;  o += pooled;
   pl->ws_klo = o;  o += pooled;
   pl->ws_vbar = o; o += pooled;
-  pl->ws_kf16 = o; o += (p->dtype == FP2_FP8_E4M3) ? pooled : 0;
   pl->ws_order = o; o += align_up(4 * (pl->nseg > 0 ? pl->nseg : 1), 1024);
   pl->ws_hist = o;  o += align_up(4 * ((int64_t)p->num_kv_heads * kCountBuckets + 1), 1024);
   pl->ws_bytes = o;
@@ -273,13 +272,12 @@ static fp2_status launch_pool(fp2_plan* pl, const void* k, const void* v, const 
   __nv_bfloat16* khi = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_khi);
   __nv_bfloat16* klo = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_klo);
   __nv_bfloat16* vb = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_vbar);
-  __half* kf16 = reinterpret_cast<__half*>(ws + pl->ws_kf16);
   if (pl->dev.fp8)
     pool_kv_kernel<true><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, lk, pl->d_blk_off, ks, vs,
-                                               pl->dev, khi, klo, vb, kf16);
+                                               pl->dev, khi, klo, vb);
   else
     pool_kv_kernel<false><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, lk, pl->d_blk_off, ks, vs,
-                                                pl->dev, khi, klo, vb, kf16);
+                                                pl->dev, khi, klo, vb);
   pl->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
@@ -352,7 +350,7 @@ static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, cons
   CUtensorMap mk, mv, mkb, mvb;
   if (!make_map(pl, &mk, k, slots, pl->prm.num_kv_heads, pl->prm.page_size, fp8) ||
       !make_map(pl, &mv, v, slots, pl->prm.num_kv_heads, pl->prm.page_size, fp8) ||
-      !make_map(pl, &mkb, ws + (fp8 ? pl->ws_kf16 : pl->ws_khi), pl->nblk_tot, pl->prm.num_kv_heads, 128, false) ||
+      !make_map(pl, &mkb, ws + pl->ws_khi, pl->nblk_tot, pl->prm.num_kv_heads, 128, false) ||
       !make_map(pl, &mvb, ws + pl->ws_vbar, pl->nblk_tot, pl->prm.num_kv_heads, 128, false))
     return FP2_ERR_CUDA;
   AttnArgs a;

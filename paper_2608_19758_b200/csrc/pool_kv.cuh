@@ -6,9 +6,9 @@
 //   kbar_hi = bf16(mean k), kbar_lo = bf16(mean k - kbar_hi)   (hi + lo carries ~16 mantissa bits for the scorer)
 //   vbar    = bf16(mean v)
 // kbar_hi and vbar double as the operands of the correction chunks in the attention kernel.
-// FP8 inputs: kbar_hi / kbar_lo hold the de-scaled mean (mean of raw values x k_scale); the attention kernel
-// runs its MMAs on F16 copies of the raw e4m3 values, so for its correction chunks this kernel also writes
-// kbar_f16 = f16(de-scaled mean k) and stores vbar as f16(mean of RAW v) -- v_scale is applied to the output.
+// FP8 inputs: the three arrays hold F16 instead of BF16 (both kernels downstream run their MMAs on F16 copies
+// of the raw e4m3 values): kbar_hi / kbar_lo = F16 pair of the de-scaled mean (mean of raw values x k_scale),
+// vbar = f16(mean of RAW v) -- v_scale is applied to the attention output.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -51,8 +51,7 @@ __global__ void __launch_bounds__(256) pool_kv_kernel(const uint8_t* __restrict_
                                                       const float* __restrict__ v_scale, DevParams P,
                                                       __nv_bfloat16* __restrict__ kbar_hi,
                                                       __nv_bfloat16* __restrict__ kbar_lo,
-                                                      __nv_bfloat16* __restrict__ vbar,
-                                                      __half* __restrict__ kbar_f16) {
+                                                      __nv_bfloat16* __restrict__ vbar) {
   constexpr int ROW_BYTES = FP8 ? 128 : 256;
   constexpr int CHUNKS = ROW_BYTES / 16;       // 16-byte chunks per token row
   constexpr int EPC = FP8 ? 16 : 8;            // elements per chunk
@@ -111,14 +110,22 @@ __global__ void __launch_bounds__(256) pool_kv_kernel(const uint8_t* __restrict_
   float mean = s / (float)ntok;
   if constexpr (FP8) mean *= (which == 0 ? k_scale[h] : 1.0f);
   const size_t o = ((size_t)gblk * P.num_kv_heads + h) * kHeadDim + c;
-  const __nv_bfloat16 hi16 = __float2bfloat16_rn(mean);
-  if (which == 0) {
-    kbar_hi[o] = hi16;
-    kbar_lo[o] = __float2bfloat16_rn(mean - __bfloat162float(hi16));
-    if constexpr (FP8) kbar_f16[o] = __float2half_rn(mean);
+  if constexpr (FP8) {
+    const __half hi16 = __float2half_rn(mean);
+    if (which == 0) {
+      reinterpret_cast<__half*>(kbar_hi)[o] = hi16;
+      reinterpret_cast<__half*>(kbar_lo)[o] = __float2half_rn(mean - __half2float(hi16));
+    } else {
+      reinterpret_cast<__half*>(vbar)[o] = hi16;
+    }
   } else {
-    if constexpr (FP8) reinterpret_cast<__half*>(vbar)[o] = __float2half_rn(mean);
-    else vbar[o] = hi16;
+    const __nv_bfloat16 hi16 = __float2bfloat16_rn(mean);
+    if (which == 0) {
+      kbar_hi[o] = hi16;
+      kbar_lo[o] = __float2bfloat16_rn(mean - __bfloat162float(hi16));
+    } else {
+      vbar[o] = hi16;
+    }
   }
 }
 

@@ -11,7 +11,8 @@
 // B = the query tile (columns), so that each consumer thread owns one pooled key and the sum over the tile's
 // rows is a sum over its own TMEM columns -- no cross-thread reduction in the main loop.  kbar enters as a
 // BF16 (hi, lo) pair accumulated into the same fp32 accumulator, which keeps the energies accurate to ~1e-5
-// relative; a single BF16 kbar would move them by ~3e-3 and flip list entries.
+// relative; a single BF16 kbar would move them by ~3e-3 and flip list entries.  FP8 inputs: the query tile is
+// widened to F16 (exact) and kbar is an F16 (hi, lo) pair.
 //
 // Roles: warps 0-3 / 4-7 = two consumer warpgroups alternating over chunks (TMEM accumulators 0 / 1) and doing
 // the selection of their tile together; warp 8 = TMA producer of kbar pieces; warp 9 = UMMA issuer; warps 10-11
@@ -27,10 +28,11 @@ namespace fp2 {
 
 constexpr int kScoreThreads = 384;
 constexpr int kScoreInfoSlots = 4;       // segment descriptors in flight
-constexpr int kScoreQBufs = 3;           // query tiles in flight: two loading while one is multiplied (one tile in
-                                         // flight per SM cannot cover the HBM latency-bandwidth product)
+constexpr int kScoreQSlots = 3;           // 32 KB query slots.  BF16: three tiles in flight (two loading while one is
+                                         // multiplied; one tile in flight per SM cannot cover the HBM latency-
+                                         // bandwidth product).  FP8: two F16 tiles + two raw 16 KB staging tiles.
 constexpr int kScoreStages = 3;          // ring of 32 KB pieces: the kbar_hi or the kbar_lo half of a 128-block chunk
-constexpr int kScoreSmemBytes = 1024 /*align*/ + kScoreQBufs * 32768 + kScoreStages * 32768 + kMaxBlocks * 4 + 2048;
+constexpr int kScoreSmemBytes = 1024 /*align*/ + kScoreQSlots * 32768 + kScoreStages * 32768 + kMaxBlocks * 4 + 2048;
 
 // Query tile -> shared memory in the K-major 128-byte-swizzled layout the UMMA descriptors expect:
 // BF16: two 64-column halves of [128 rows x 128 B]; FP8 is widened to BF16 on the way (exact).
@@ -74,6 +76,46 @@ __device__ __forceinline__ void load_q_tile_bf16(uint8_t* sQ, const uint8_t* __r
       if (i < kTileRows * 16)
         *reinterpret_cast<uint4*>(sQ + (ch >> 3) * 16384 + sw128_offset(row, ch & 7)) = v[u];
     }
+  }
+}
+
+// One raw FP8 tile (128 rows x 128 bytes, 128-byte swizzle as TMA wrote it) -> one F16 tile in the two-halves
+// layout of the K / V rings.  nthr threads (a multiple of 8); eight consecutive threads take one row, so every quarter-warp reads
+// one whole 128-byte row (conflict-free).  Element order inside a row is preserved, so the same routine
+// serves K (K-major operand) and V (MN-major operand).
+__device__ __forceinline__ void widen_tile_f16(const uint8_t* raw, uint8_t* dst, int t, int nthr) {
+#pragma unroll 4
+  for (int i = t; i < kTileRows * 8; i += nthr) {
+    const int row = i >> 3, c = i & 7;        // c: 16-byte chunk = 16 elements d = 16c .. 16c+15
+    const uint4 v = *reinterpret_cast<const uint4*>(raw + sw128_offset(row, c));
+    const uint4 lo = make_uint4(e4m3x2_to_f16x2(v.x), e4m3x2_to_f16x2(v.x >> 16), e4m3x2_to_f16x2(v.y),
+                                e4m3x2_to_f16x2(v.y >> 16));
+    const uint4 hi = make_uint4(e4m3x2_to_f16x2(v.z), e4m3x2_to_f16x2(v.z >> 16), e4m3x2_to_f16x2(v.w),
+                                e4m3x2_to_f16x2(v.w >> 16));
+    uint8_t* half = dst + (c >> 2) * 16384;   // d < 64 -> first half
+    const int oc = (c & 3) * 2;               // chunk index inside the half (8 f16 per 16 bytes)
+    *reinterpret_cast<uint4*>(half + sw128_offset(row, oc)) = lo;
+    *reinterpret_cast<uint4*>(half + sw128_offset(row, oc + 1)) = hi;
+  }
+}
+
+// Raw FP8 query tile -> shared memory with cp.async in the layout widen_tile_f16 reads (128-byte rows, swizzled).
+__device__ __forceinline__ void load_q_raw_async(uint8_t* sRaw, const uint8_t* __restrict__ q, const SegInfo& sg,
+                                                 const DevParams& P, int t, int nthr) {
+  const int g = P.group;
+  const uint32_t base = smem_u32(sRaw);
+  for (int i = t; i < kTileRows * 8; i += nthr) {
+    const int row = i >> 3, ch = i & 7;
+    const uint8_t* src = q;
+    uint32_t nbytes = 0;
+    if (row < sg.nrows) {
+      const int r = sg.r0 + row;
+      const size_t tok = (size_t)sg.q_tok0 + r / g;
+      const size_t head = (size_t)sg.h * g + r % g;
+      src = q + (tok * P.num_q_heads + head) * kHeadDim + ch * 16;
+      nbytes = 16;
+    }
+    cp_async16(base + sw128_offset(row, ch), src, nbytes);
   }
 }
 
@@ -142,14 +184,16 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
                     int32_t* __restrict__ blk_idx, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem;                                    // kScoreQBufs x 32 KB query tiles
-  uint8_t* sStage = smem + kScoreQBufs * 32768;                    // kScoreStages x 32 KB pieces (kbar_hi or kbar_lo chunk)
+  constexpr int kScoreQBufs = FP8 ? 2 : 3;
+  uint8_t* sQ = smem;                                    // kScoreQBufs x 32 KB query tiles (+ raw staging, FP8)
+  uint8_t* sQraw = smem + 2 * 32768;                     // FP8: two raw e4m3 tiles of 16 KB
+  uint8_t* sStage = smem + kScoreQSlots * 32768;                    // kScoreStages x 32 KB pieces (kbar_hi or kbar_lo chunk)
   float* sE = reinterpret_cast<float*>(sStage + kScoreStages * 32768);  // per candidate: log2 of its energy
   float* sC = sE + kMaxBlocks;                                          // [kScoreQBufs][128] per-row multiplier (FP8)
 
   __shared__ SegInfo info[kScoreInfoSlots];
   __shared__ int info_valid[kScoreInfoSlots];
-  __shared__ uint64_t info_full[kScoreInfoSlots], info_empty[kScoreInfoSlots], q_full[kScoreQBufs], q_empty[kScoreQBufs];
+  __shared__ uint64_t info_full[kScoreInfoSlots], info_empty[kScoreInfoSlots], q_full[kScoreQSlots], q_empty[kScoreQSlots];
   __shared__ uint64_t full[kScoreStages], empty[kScoreStages], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
@@ -207,13 +251,12 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       if (t64 == 0) mbar_arrive(&info_full[slot]);
       if (!valid) return false;
       const SegInfo sg = info[slot];
-      // the Q buffer is free once every MMA of the tile that used it kScoreQBufs tiles ago has completed
-      if (k >= kScoreQBufs) mbar_wait(&q_empty[qb], ((k / kScoreQBufs) - 1) & 1, ctx, 112);
       if constexpr (FP8) {
-        load_q_tile_bf16<true, 8>(sQ + qb * 32768, q, sg, P, t64, 64);
-        for (int j = t64; j < kTileRows; j += 64)
-          sC[qb * 128 + j] = P.scale_log2 * q_scale[sg.h * P.group + (sg.r0 + j) % P.group];
+        // raw e4m3 tile into the staging slot (its previous content was widened two tiles ago by these threads)
+        load_q_raw_async(sQraw + (k & 1) * 16384, q, sg, P, t64, 64);
       } else {
+        // the Q buffer is free once every MMA of the tile that used it kScoreQBufs tiles ago has completed
+        if (k >= kScoreQBufs) mbar_wait(&q_empty[qb], ((k / kScoreQBufs) - 1) & 1, ctx, 112);
         load_q_tile_async(sQ + qb * 32768, q, sg, P, t64, 64, false);
       }
       cp_async_commit();
@@ -223,8 +266,17 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
     for (int k = 0; have; ++k) {
       const bool next = issue(k + 1);
       if (next) cp_async_wait_group<1>(); else cp_async_wait_group<0>();
+      const int qb = k % kScoreQBufs;
+      if constexpr (FP8) {
+        named_bar_sync(2, 64);   // every thread's copies of tile k have landed
+        if (k >= kScoreQBufs) mbar_wait(&q_empty[qb], ((k / kScoreQBufs) - 1) & 1, ctx, 113);
+        widen_tile_f16(sQraw + (k & 1) * 16384, sQ + qb * 32768, t64, 64);
+        const SegInfo& sgk = info[k % kScoreInfoSlots];
+        for (int j = t64; j < kTileRows; j += 64)
+          sC[qb * 128 + j] = P.scale_log2 * q_scale[sgk.h * P.group + (sgk.r0 + j) % P.group];
+      }
       fence_proxy_async();
-      mbar_arrive(&q_full[k % kScoreQBufs]);
+      mbar_arrive(&q_full[qb]);
       have = next;
     }
   } else if (warp == 8) {
@@ -257,7 +309,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
   } else if (warp == 9) {
     // ---------------- UMMA issuer: acc[c & 1] = kbar_hi Q^T + kbar_lo Q^T ----------------
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(128, 128, 1, 1, 0, 0);
+      constexpr uint32_t idesc = FP8 ? make_idesc(128, 128, 0, 0, 0, 0) : make_idesc(128, 128, 1, 1, 0, 0);
       uint32_t pc = 0, ac0 = 0, ac1 = 0;
       for (int it = 0;; ++it) {
         const int slot = it % kScoreInfoSlots, qb = it % kScoreQBufs;

@@ -169,27 +169,6 @@ __device__ __forceinline__ void load_q_tile_f16(uint8_t* sQ, const uint8_t* __re
   }
 }
 
-// One raw FP8 tile (128 rows x 128 bytes, 128-byte swizzle as TMA wrote it) -> one F16 tile in the two-halves
-// layout of the K / V rings.  128 threads; eight consecutive threads take one row, so every quarter-warp reads
-// one whole 128-byte row (conflict-free).  Element order inside a row is preserved, so the same routine
-// serves K (K-major operand) and V (MN-major operand).
-__device__ __forceinline__ void widen_tile_f16(const uint8_t* raw, uint8_t* dst, int t) {
-#pragma unroll
-  for (int k = 0; k < 8; ++k) {
-    const int i = t + 128 * k;
-    const int row = i >> 3, c = i & 7;        // c: 16-byte chunk = 16 elements d = 16c .. 16c+15
-    const uint4 v = *reinterpret_cast<const uint4*>(raw + sw128_offset(row, c));
-    const uint4 lo = make_uint4(e4m3x2_to_f16x2(v.x), e4m3x2_to_f16x2(v.x >> 16), e4m3x2_to_f16x2(v.y),
-                                e4m3x2_to_f16x2(v.y >> 16));
-    const uint4 hi = make_uint4(e4m3x2_to_f16x2(v.z), e4m3x2_to_f16x2(v.z >> 16), e4m3x2_to_f16x2(v.w),
-                                e4m3x2_to_f16x2(v.w >> 16));
-    uint8_t* half = dst + (c >> 2) * 16384;   // d < 64 -> first half
-    const int oc = (c & 3) * 2;               // chunk index inside the half (8 f16 per 16 bytes)
-    *reinterpret_cast<uint4*>(half + sw128_offset(row, oc)) = lo;
-    *reinterpret_cast<uint4*>(half + sw128_offset(row, oc + 1)) = hi;
-  }
-}
-
 template <bool FP8>
 __global__ void __launch_bounds__(AttnCfg<FP8>::kThreads, 1)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
@@ -273,7 +252,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
             uint64_t* d_full = kv ? &v_full[ds] : &k_full[ds];
             if (dc >= (uint32_t)dn) mbar_wait(d_empty, ((dc / dn) - 1) & 1, ctx, 602);
             mbar_wait(&raw_full[rs], (rc / kNRaw) & 1, ctx, 603);
-            widen_tile_f16(sRaw + rs * kRawBytes, (kv ? sV : sK) + ds * kTileBytes, t128);
+            widen_tile_f16(sRaw + rs * kRawBytes, (kv ? sV : sK) + ds * kTileBytes, t128, 128);
             fence_proxy_async();
             named_bar_sync(3, 128);
             if (t128 == 0) {
