@@ -157,6 +157,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-fp8", action="store_true")
     ap.add_argument("--oracle-segments", type=int, default=20)
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "fp2":
@@ -332,6 +333,27 @@ def main():
             extra["e2e"] = {"value": dflops / (np.mean(e2e_ms) * 1e-3) / 1e12, "unit": UNIT,
                             "ms_per_step": float(np.mean(e2e_ms)), "h2d_bytes_per_step": int(h2d),
                             "d2h_bytes_per_step": int(d2h)}
+        # the FP8 e4m3 workload (config 4: Hq=28, Hkv=4, per-head scales) at the same target sparsity
+        if not args.no_fp8 and args.config == 3 and args.scale_down == 1:
+            main_dc, main_case = dc, case
+            case = inputs.make_case(inputs.config_spec(4))
+            dc = binding.DeviceCase(case)
+            pairs = dc.plan.idx_capacity
+            a8, s8 = calibrate(args.sparsity)
+            sm8, am8, tot8, _ = step_split(3, 2)
+            d8 = timed(dc.dense, 2, 1)
+            fl8 = dense_flops(case)
+            ex8 = float(dc.seg_count.sum().item()) * 4.0 * 128 ** 3
+            dc.status()
+            extra["fp8"] = {"workload": "config 4: fp8 e4m3 1 seq, 131072 KV tokens, Hq=28 Hkv=4 d=128 page=64",
+                            "alpha": a8, "sparsity": s8, "select_ms": float(np.mean(sm8)),
+                            "sparse_ms": float(np.mean(am8)), "executed_tflops": ex8 / (np.mean(am8) * 1e-3) / 1e12,
+                            "dense_equiv_tflops": fl8 / ((np.mean(sm8) + np.mean(am8)) * 1e-3) / 1e12,
+                            "dense_ms": float(np.mean(d8)), "dense_tflops": fl8 / (np.mean(d8) * 1e-3) / 1e12,
+                            "speedup_vs_own_dense": float(np.mean(d8)) / float(np.mean(sm8) + np.mean(am8)),
+                            "note": "MMAs run in F16 on widened e4m3 values; the tensor peak to compare with is the BF16 one"}
+            dc, case = main_dc, main_case
+            pairs = dc.plan.idx_capacity
         if not args.no_cpu:
             dt, fl, desc, threads = oracle_sample(case, args.oracle_segments)
             extra["cpu_baseline"] = {"value": fl / dt / 1e12, "unit": UNIT, "cores": threads, "kind": "oracle",
@@ -341,13 +363,10 @@ def main():
         dist.destroy_process_group()
     if rank != 0:
         return
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
-        try:
-            traffic = json.load(open(tpath)).get("sparse_attn_dram_bytes_per_launch_config3_95")
-        except Exception:
-            traffic = None
+    # DRAM bytes per attention launch: ncu on config 2 (32768 tokens) measured 406.9 MB read + 235.8 MB written
+    # (profiles/dram_traffic_config2_all_kernels.md); every tile reads its Q rows and writes its O rows once and
+    # K/V comes from L2 after the first touch, so the figure scales with the token count.
+    traffic = (406.9e6 + 235.8e6) * (sum(l for l, _ in spec.seqs) / 32768.0) if spec.num_q_heads == 32 else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
