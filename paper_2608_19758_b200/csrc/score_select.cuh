@@ -131,25 +131,38 @@ __device__ __forceinline__ void score_chunk(uint32_t lane_addr, float cs, const 
   tmem_wait_ld();
   tc_fence_before();
   mbar_arrive(acc_empty_bar);
+  // x_j = s_j * multiplier (packed fp32x2), rows past nrows masked to -inf
   float x[128];
 #pragma unroll
-  for (int j = 0; j < 128; ++j) {
-    float mult = cs;
-    if constexpr (FP8) mult = sC[j];
-    x[j] = __uint_as_float(xv[j]) * mult;
-    if constexpr (PARTIAL) x[j] = (j < nrows) ? x[j] : -INFINITY;
+  for (int j = 0; j < 128; j += 2) {
+    uint64_t mult2 = f2_pack(cs, cs);
+    if constexpr (FP8) mult2 = f2_pack(sC[j], sC[j + 1]);
+    f2_unpack(f2_mul(f2_pack(__uint_as_float(xv[j]), __uint_as_float(xv[j + 1])), mult2), x[j], x[j + 1]);
+    if constexpr (PARTIAL) {
+      x[j] = (j < nrows) ? x[j] : -INFINITY;
+      x[j + 1] = (j + 1 < nrows) ? x[j + 1] : -INFINITY;
+    }
   }
   float m8[8];
 #pragma unroll
-  for (int j = 0; j < 8; ++j) m8[j] = x[j];
+  for (int c = 0; c < 8; ++c) {
+    const float* v = &x[c * 16];
+    m8[c] = max3(max3(max3(v[0], v[1], v[2]), max3(v[3], v[4], v[5]), max3(v[6], v[7], v[8])),
+                 max3(v[9], v[10], v[11]), max3(max3(v[12], v[13], v[14]), v[15], v[15]));
+  }
+  const float m = fmaxf(max3(m8[0], m8[1], m8[2]), max3(max3(m8[3], m8[4], m8[5]), m8[6], m8[7]));
+  const uint64_t nm2 = f2_pack(-m, -m);
+  uint64_t s4[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
-  for (int j = 8; j < 128; ++j) m8[j & 7] = fmaxf(m8[j & 7], x[j]);
-  const float m = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])), fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
-  float s8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-  for (int j = 0; j < 128; ++j) s8[j & 7] += ex2(x[j] - m);
+  for (int j = 0; j < 128; j += 2) {
+    float d0, d1;
+    f2_unpack(f2_add(f2_pack(x[j], x[j + 1]), nm2), d0, d1);
+    s4[(j >> 1) & 3] = f2_add(s4[(j >> 1) & 3], f2_pack(ex2(d0), ex2(d1)));
+  }
+  float t0, t1;
+  f2_unpack(f2_add(f2_add(s4[0], s4[1]), f2_add(s4[2], s4[3])), t0, t1);
   m_out = m;
-  sum_out = ((s8[0] + s8[1]) + (s8[2] + s8[3])) + ((s8[4] + s8[5]) + (s8[6] + s8[7]));
+  sum_out = t0 + t1;
 }
 
 // BF16 query tile -> shared memory with cp.async: every 16-byte piece of the tile is in flight at once (the

@@ -98,7 +98,8 @@ __device__ __forceinline__ void mask_half(uint32_t s_addr, int col0, int tok_lim
   tmem_wait_st();
 }
 
-// Row maximum of this thread's 64 logit columns (raw, unscaled): two TMEM loads in flight, eight max chains.
+// Row maximum of this thread's 64 logit columns (raw, unscaled): two TMEM loads in flight, eight chains of
+// three-input maxima.
 __device__ __forceinline__ float half_row_max(uint32_t s_addr) {
   uint32_t sv[64];
   tmem_ld32(s_addr, reinterpret_cast<uint32_t(&)[32]>(sv[0]));
@@ -106,17 +107,20 @@ __device__ __forceinline__ float half_row_max(uint32_t s_addr) {
   tmem_wait_ld();
   float mx8[8];
 #pragma unroll
-  for (int c = 0; c < 8; ++c) mx8[c] = __uint_as_float(sv[c]);
-#pragma unroll
-  for (int j = 8; j < 64; ++j) mx8[j & 7] = fmaxf(mx8[j & 7], __uint_as_float(sv[j]));
-  return fmaxf(fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3])), fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+  for (int c = 0; c < 8; ++c) {
+    const float* v = reinterpret_cast<const float*>(&sv[c * 8]);
+    mx8[c] = fmaxf(max3(max3(v[0], v[1], v[2]), v[3], v[4]), max3(v[5], v[6], v[7]));
+  }
+  return fmaxf(max3(mx8[0], mx8[1], mx8[2]), max3(max3(mx8[3], mx8[4], mx8[5]), mx8[6], mx8[7]));
 }
 
-// p = 2^(s * cs + neg_m) for this thread's 64 columns, written as BF16 pairs to 32 columns at p_addr.
-// The second TMEM load is in flight while the first half is exponentiated.  Returns the row's partial sum.
+// p = 2^(s * cs + neg_m) for this thread's 64 columns, written as 16-bit pairs to 32 columns at p_addr.
+// The second TMEM load is in flight while the first half is exponentiated.  Scaling and row sum use packed
+// fp32x2 instructions.  Returns the row's partial sum.
 template <bool F16>
 __device__ __forceinline__ float half_row_exp(uint32_t s_addr, uint32_t p_addr, float cs, float neg_m) {
-  float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+  const uint64_t cs2 = f2_pack(cs, cs), nm2 = f2_pack(neg_m, neg_m);
+  uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};   // four independent (lo, hi) accumulators, +0.0f bit patterns
   uint32_t buf[2][32];
   tmem_ld32(s_addr, buf[0]);
   tmem_wait_ld();
@@ -126,15 +130,20 @@ __device__ __forceinline__ float half_row_exp(uint32_t s_addr, uint32_t p_addr, 
     uint32_t pk[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      const float p0 = ex2(fmaf(__uint_as_float(buf[k][2 * j]), cs, neg_m));
-      const float p1 = ex2(fmaf(__uint_as_float(buf[k][2 * j + 1]), cs, neg_m));
-      sum4[j & 3] += p0 + p1;
+      const uint64_t x2 = f2_fma(f2_pack(__uint_as_float(buf[k][2 * j]), __uint_as_float(buf[k][2 * j + 1])), cs2, nm2);
+      float x0, x1;
+      f2_unpack(x2, x0, x1);
+      const float p0 = ex2(x0), p1 = ex2(x1);
+      sum2[j & 3] = f2_add(sum2[j & 3], f2_pack(p0, p1));
       pk[j] = F16 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1);
     }
     if (k == 0) tmem_wait_ld();
     tmem_st16(p_addr + k * 16, pk);
   }
-  return (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+  float a0, a1, b0, b1;
+  f2_unpack(f2_add(f2_add(sum2[0], sum2[1]), f2_add(sum2[2], sum2[3])), a0, a1);
+  (void)b0; (void)b1;
+  return a0 + a1;
 }
 
 // FP8 query tile -> shared memory as F16 (exact), same K-major swizzled layout as the BF16 tile.
