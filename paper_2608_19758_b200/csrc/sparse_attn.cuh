@@ -42,10 +42,12 @@ constexpr int kRawBytes = 16384;    // one 128 x 128 tile of FP8 elements as TMA
 template <bool FP8>
 struct AttnCfg {
   static constexpr int kThreads = FP8 ? 512 : 384;
-  static constexpr int kNK = FP8 ? 2 : 3;   // K ring stages (32 KB each)
+  static constexpr int kNQ = FP8 ? 1 : 2;   // Q tiles in shared memory: two let the next unit's queries land while
+                                            // this unit is still being multiplied (FP8 has no room for a second)
+  static constexpr int kNK = 2;             // K ring stages (32 KB each)
   static constexpr int kNV = 2;             // V ring stages
   static constexpr int kNRaw = FP8 ? 3 : 0; // raw FP8 tile ring (16 KB each), K and V tiles alternate
-  static constexpr int kSmemBytes = 1024 + kTileBytes * (1 + kNK + kNV) + kNRaw * kRawBytes + 3072;
+  static constexpr int kSmemBytes = 1024 + kTileBytes * (kNQ + kNK + kNV) + kNRaw * kRawBytes + 3072;
   static constexpr int kFmt = FP8 ? 0 : 1;  // UMMA kind::f16 operand format: 0 = F16, 1 = BF16
 };
 
@@ -183,19 +185,19 @@ __global__ void __launch_bounds__(AttnCfg<FP8>::kThreads, 1)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                    const __grid_constant__ CUtensorMap map_kbar, const __grid_constant__ CUtensorMap map_vbar,
                    AttnArgs A, DevParams P) {
-  constexpr int kNK = AttnCfg<FP8>::kNK, kNV = AttnCfg<FP8>::kNV, kNRaw = AttnCfg<FP8>::kNRaw;
+  constexpr int kNQ = AttnCfg<FP8>::kNQ, kNK = AttnCfg<FP8>::kNK, kNV = AttnCfg<FP8>::kNV, kNRaw = AttnCfg<FP8>::kNRaw;
   constexpr int kAttnThreads = AttnCfg<FP8>::kThreads;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = smem;
-  uint8_t* sK = smem + kTileBytes;
+  uint8_t* sK = smem + kNQ * kTileBytes;
   uint8_t* sV = sK + kNK * kTileBytes;
   uint8_t* sRaw = sV + kNV * kTileBytes;                          // FP8 only: raw tile ring
   float* sX = reinterpret_cast<float*>(sRaw + kNRaw * kRawBytes);  // [2 parity][2 wg][128] row-max / row-sum exchange
 
   __shared__ TileInfo info[2];
   __shared__ uint32_t sel_bits[2][kMaxBlocks / 32];
-  __shared__ uint64_t info_full[2], info_empty[2], q_full, q_empty, tile_done;
+  __shared__ uint64_t info_full[2], info_empty[2], q_full[2], q_empty[2], tile_done;
   __shared__ uint64_t k_full[kNK], k_empty[kNK], v_full[kNV], v_empty[kNV];
   __shared__ uint64_t s_full[2], p_ready[2], o_done;
   __shared__ uint64_t raw_full[kNRaw > 0 ? kNRaw : 1], raw_empty[kNRaw > 0 ? kNRaw : 1];
@@ -213,8 +215,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       mbar_init(&s_full[i], 1);
       mbar_init(&p_ready[i], 256);
     }
-    mbar_init(&q_full, 64);
-    mbar_init(&q_empty, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&q_full[i], 64); mbar_init(&q_empty[i], 1); }
     mbar_init(&tile_done, 1);
     mbar_init(&o_done, 1);
     for (int i = 0; i < kNK; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
@@ -342,12 +343,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       named_bar_sync(2, 64);
       if (t64 == 0) mbar_arrive(&info_full[slot]);
       if (!valid) break;
-      // Q tile: wait until every S = Q K^T of the previous unit has completed, then overwrite
-      if (it >= 1) mbar_wait(&q_empty, (it - 1) & 1, ctx, 202);
-      if constexpr (FP8) load_q_tile_f16(sQ, A.q, ti.sg, P, t64, 64);
-      else load_q_tile_async(sQ, A.q, ti.sg, P, t64, 64);
+      // Q tile: wait until every S = Q K^T of the unit that last used this buffer has completed, then overwrite
+      const int qb = it % kNQ;
+      if (it >= kNQ) mbar_wait(&q_empty[qb], ((it / kNQ) - 1) & 1, ctx, 202);
+      if constexpr (FP8) load_q_tile_f16(sQ + qb * kTileBytes, A.q, ti.sg, P, t64, 64);
+      else load_q_tile_async(sQ + qb * kTileBytes, A.q, ti.sg, P, t64, 64);
       fence_proxy_async();
-      mbar_arrive(&q_full);
+      mbar_arrive(&q_full[qb]);
     }
   } else if (warp == 8) {
     // =============================== TMA producer ===============================
@@ -449,7 +451,6 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       constexpr int kFmt = AttnCfg<FP8>::kFmt;
       constexpr uint32_t idesc_qk = make_idesc(128, 128, kFmt, kFmt, 0, 0);
       constexpr uint32_t idesc_pv = make_idesc(128, 128, kFmt, kFmt, 0, 1);
-      const uint32_t q_addr = smem_u32(sQ);
       uint32_t kc = 0, vc = 0, pc0 = 0, pc1 = 0;
       auto issue_pv = [&](int j) {
         const int b = j & 1;
@@ -474,7 +475,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         const TileInfo& ti = info[slot];
         if (!ti.valid) break;
         const int n_it = ti.T + ti.nchunk;
-        mbar_wait(&q_full, it & 1, ctx, 404);
+        const int qb = it % kNQ;
+        mbar_wait(&q_full[qb], (it / kNQ) & 1, ctx, 404);
+        const uint32_t q_addr = smem_u32(sQ + qb * kTileBytes);
         for (int i = 0; i < n_it; ++i) {
           const int a = i & 1;
           const int ks_ = kc % kNK;
@@ -492,11 +495,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           umma_commit(&k_empty[ks_]);
           umma_commit(&s_full[a]);
           ++kc;
-          if (i == n_it - 1) umma_commit(&q_empty);
+          if (i == n_it - 1) umma_commit(&q_empty[qb]);
           if (i >= 1) issue_pv(i - 1);
         }
         if (n_it >= 1) issue_pv(n_it - 1);
-        else umma_commit(&q_empty);  // empty list: nothing read Q, release it at once
+        else umma_commit(&q_empty[qb]);  // empty list: nothing read Q, release it at once
         umma_commit(&tile_done);
         mbar_arrive(&info_empty[slot]);
       }
