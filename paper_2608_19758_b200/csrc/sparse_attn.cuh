@@ -47,7 +47,7 @@ struct AttnCfg {
   static constexpr int kNK = 2;             // K ring stages (32 KB each)
   static constexpr int kNV = 2;             // V ring stages
   static constexpr int kNRaw = FP8 ? 3 : 0; // raw FP8 tile ring (16 KB each), K and V tiles alternate
-  static constexpr int kSmemBytes = 1024 + kTileBytes * (kNQ + kNK + kNV) + kNRaw * kRawBytes + 3072;
+  static constexpr int kSmemBytes = 1024 + kTileBytes * (kNQ + kNK + kNV) + kNRaw * kRawBytes + 4096;
   static constexpr int kFmt = FP8 ? 0 : 1;  // UMMA kind::f16 operand format: 0 = F16, 1 = BF16
 };
 
@@ -604,7 +604,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       // ------------------------------ epilogue ------------------------------
       mbar_wait(&tile_done, it & 1, ctx, 503);
       tc_fence_after();
-      float* xch = sX + 512;
+      float* xch = sX + 512 + (it & 1) * 256;   // by tile parity: no barrier is needed before its next use
       xch[wg * 128 + row] = l;
       named_bar_sync(1, 256);
       const float L = l + xch[(wg ^ 1) * 128 + row];
@@ -628,16 +628,14 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           const float v1 = have_o ? __uint_as_float(a0[2 * j + 1]) * inv : 0.f;
           o[j] = pack_bf16x2(v0, v1);
         }
-        if (row_ok) {
-          uint4* dst = reinterpret_cast<uint4*>(orow + k * 32);
-#pragma unroll
-          for (int j = 0; j < 4; ++j) dst[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
+        if (row_ok) {   // 32-byte stores: every instruction writes whole sectors
+          st_global_v8(orow + k * 32, &o[0]);
+          st_global_v8(orow + k * 32 + 16, &o[8]);
         }
       }
       if (wg == 0 && row_ok && A.lse != nullptr)
         A.lse[(size_t)head * P.total_q + tok] = (m + log2f(L)) * 0.6931471805599453f;
       tc_fence_before();
-      named_bar_sync(1, 256);   // the exchange buffers are reused by the next tile
       mbar_arrive(&info_empty[slot]);
     }
   }
