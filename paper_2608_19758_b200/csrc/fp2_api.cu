@@ -78,7 +78,7 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
     ntiles_tot += (g * lq + kTileRows - 1) / kTileRows;
     nblk_tot += nblk;
   }
-  if (ntiles_tot * p->num_kv_heads > (int64_t)0x7fffffff || nblk_tot * p->num_kv_heads > (int64_t)0x7fffffff)
+  if (ntiles_tot * p->num_kv_heads > (int64_t)0x7fffffff || nblk_tot * p->num_kv_heads * 2 > (int64_t)0x7fffffff)
     return FP2_ERR_CAPACITY;
 
   fp2_plan* pl = new (std::nothrow) fp2_plan();
@@ -268,7 +268,7 @@ static fp2_status check_common(fp2_plan* pl, const void* q, const void* k, const
 static fp2_status launch_pool(fp2_plan* pl, const void* k, const void* v, const int32_t* pt, const int32_t* lk,
                               const float* ks, const float* vs, uint8_t* ws, cudaStream_t st) {
   if (pl->nblk_tot == 0) return FP2_OK;
-  const unsigned grid = (unsigned)(pl->nblk_tot * pl->prm.num_kv_heads);
+  const unsigned grid = (unsigned)(pl->nblk_tot * pl->prm.num_kv_heads * 2);   // K and V pooled by separate CTAs
   __nv_bfloat16* khi = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_khi);
   __nv_bfloat16* klo = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_klo);
   __nv_bfloat16* vb = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_vbar);

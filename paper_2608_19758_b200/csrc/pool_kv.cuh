@@ -39,28 +39,32 @@ __device__ __forceinline__ void accum16(const uint4& v, float* acc) {
   }
 }
 
-// 1-D grid of nblk_tot * Hkv CTAs, KV head fastest: CTAs that run together read neighbouring heads of the same
-// tokens, i.e. whole contiguous token rows of the cache.  256 threads.
+// 1-D grid of nblk_tot * Hkv * 2 CTAs: (K or V) fastest, then the KV head, then the block, so CTAs that run
+// together read neighbouring pieces of the same token rows.  One CTA pools one operand of one (block, head):
+// 128 token rows of 256 B (BF16) / 128 B (FP8).  256 threads, every load of a thread issued before the first
+// use; small enough in registers for four CTAs per SM, which is what hides the page-table -> data dependency.
 template <bool FP8>
-__global__ void __launch_bounds__(256) pool_kv_kernel(const uint8_t* __restrict__ k_cache,
-                                                      const uint8_t* __restrict__ v_cache,
-                                                      const int32_t* __restrict__ page_table,
-                                                      const int32_t* __restrict__ seqlens_k,
-                                                      const int32_t* __restrict__ blk_off,  // [ns+1]
-                                                      const float* __restrict__ k_scale,
-                                                      const float* __restrict__ v_scale, DevParams P,
-                                                      __nv_bfloat16* __restrict__ kbar_hi,
-                                                      __nv_bfloat16* __restrict__ kbar_lo,
-                                                      __nv_bfloat16* __restrict__ vbar) {
+__global__ void __launch_bounds__(256, 4) pool_kv_kernel(const uint8_t* __restrict__ k_cache,
+                                                         const uint8_t* __restrict__ v_cache,
+                                                         const int32_t* __restrict__ page_table,
+                                                         const int32_t* __restrict__ seqlens_k,
+                                                         const int32_t* __restrict__ blk_off,  // [ns+1]
+                                                         const float* __restrict__ k_scale,
+                                                         const float* __restrict__ v_scale, DevParams P,
+                                                         __nv_bfloat16* __restrict__ kbar_hi,
+                                                         __nv_bfloat16* __restrict__ kbar_lo,
+                                                         __nv_bfloat16* __restrict__ vbar) {
   constexpr int ROW_BYTES = FP8 ? 128 : 256;
   constexpr int CHUNKS = ROW_BYTES / 16;       // 16-byte chunks per token row
   constexpr int EPC = FP8 ? 16 : 8;            // elements per chunk
   constexpr int ROWS_PER_PASS = 256 / CHUNKS;  // 16 (bf16) or 32 (fp8)
   constexpr int PASSES = kBlock / ROWS_PER_PASS;
 
-  __shared__ float red[2][ROWS_PER_PASS][kHeadDim + 4];
+  __shared__ float red[ROWS_PER_PASS][kHeadDim + 4];
 
-  const int gblk = blockIdx.x / P.num_kv_heads, h = blockIdx.x % P.num_kv_heads;
+  const int which = blockIdx.x & 1;            // 0: K, 1: V
+  const int bh = blockIdx.x >> 1;
+  const int gblk = bh / P.num_kv_heads, h = bh % P.num_kv_heads;
   // sequence of this pooled block: binary search in blk_off
   int lo = 0, hi = P.num_seqs;
   while (hi - lo > 1) {
@@ -73,58 +77,51 @@ __global__ void __launch_bounds__(256) pool_kv_kernel(const uint8_t* __restrict_
   const int chunk = threadIdx.x % CHUNKS, rg = threadIdx.x / CHUNKS;
   const int32_t* pt = page_table + (size_t)b * P.max_pages_per_seq;
   const size_t row_stride = (size_t)P.num_kv_heads * ROW_BYTES;
+  const uint8_t* cache = which ? v_cache : k_cache;
 
-  float ak[EPC], av[EPC];
-#pragma unroll
-  for (int i = 0; i < EPC; ++i) ak[i] = av[i] = 0.f;
-
-  uint4 kv[PASSES], vv[PASSES];
+  uint4 dv[PASSES];
 #pragma unroll
   for (int ps = 0; ps < PASSES; ++ps) {
     const int tl = ps * ROWS_PER_PASS + rg;
-    kv[ps] = make_uint4(0, 0, 0, 0);
-    vv[ps] = make_uint4(0, 0, 0, 0);
+    dv[ps] = make_uint4(0, 0, 0, 0);   // zero bit patterns add 0 in both encodings
     if (tl < ntok) {
       const int j = J * kBlock + tl;
       const size_t slot = (size_t)pt[j / P.page_size] * P.page_size + (j % P.page_size);
-      const size_t off = slot * row_stride + (size_t)h * ROW_BYTES + chunk * 16;
-      kv[ps] = __ldg(reinterpret_cast<const uint4*>(k_cache + off));
-      vv[ps] = __ldg(reinterpret_cast<const uint4*>(v_cache + off));
+      dv[ps] = __ldg(reinterpret_cast<const uint4*>(cache + slot * row_stride + (size_t)h * ROW_BYTES + chunk * 16));
     }
   }
+  float acc[EPC];
 #pragma unroll
-  for (int ps = 0; ps < PASSES; ++ps) {   // zero bit patterns add 0 in both encodings
-    accum16<FP8>(kv[ps], ak);
-    accum16<FP8>(vv[ps], av);
-  }
+  for (int i = 0; i < EPC; ++i) acc[i] = 0.f;
 #pragma unroll
-  for (int i = 0; i < EPC; ++i) {
-    red[0][rg][chunk * EPC + i] = ak[i];
-    red[1][rg][chunk * EPC + i] = av[i];
-  }
+  for (int ps = 0; ps < PASSES; ++ps) accum16<FP8>(dv[ps], acc);
+#pragma unroll
+  for (int i = 0; i < EPC; ++i) red[rg][chunk * EPC + i] = acc[i];
   __syncthreads();
-  const int which = threadIdx.x / kHeadDim, c = threadIdx.x % kHeadDim;
-  float s = 0.f;
+  if (threadIdx.x < kHeadDim) {
+    const int c = threadIdx.x;
+    float s = 0.f;
 #pragma unroll
-  for (int r = 0; r < ROWS_PER_PASS; ++r) s += red[which][r][c];
-  float mean = s / (float)ntok;
-  if constexpr (FP8) mean *= (which == 0 ? k_scale[h] : 1.0f);
-  const size_t o = ((size_t)gblk * P.num_kv_heads + h) * kHeadDim + c;
-  if constexpr (FP8) {
-    const __half hi16 = __float2half_rn(mean);
-    if (which == 0) {
-      reinterpret_cast<__half*>(kbar_hi)[o] = hi16;
-      reinterpret_cast<__half*>(kbar_lo)[o] = __float2half_rn(mean - __half2float(hi16));
+    for (int r = 0; r < ROWS_PER_PASS; ++r) s += red[r][c];
+    float mean = s / (float)ntok;
+    if constexpr (FP8) mean *= (which == 0 ? k_scale[h] : 1.0f);
+    const size_t o = ((size_t)gblk * P.num_kv_heads + h) * kHeadDim + c;
+    if constexpr (FP8) {
+      const __half hi16 = __float2half_rn(mean);
+      if (which == 0) {
+        reinterpret_cast<__half*>(kbar_hi)[o] = hi16;
+        reinterpret_cast<__half*>(kbar_lo)[o] = __float2half_rn(mean - __half2float(hi16));
+      } else {
+        reinterpret_cast<__half*>(vbar)[o] = hi16;
+      }
     } else {
-      reinterpret_cast<__half*>(vbar)[o] = hi16;
-    }
-  } else {
-    const __nv_bfloat16 hi16 = __float2bfloat16_rn(mean);
-    if (which == 0) {
-      kbar_hi[o] = hi16;
-      kbar_lo[o] = __float2bfloat16_rn(mean - __bfloat162float(hi16));
-    } else {
-      vbar[o] = hi16;
+      const __nv_bfloat16 hi16 = __float2bfloat16_rn(mean);
+      if (which == 0) {
+        kbar_hi[o] = hi16;
+        kbar_lo[o] = __float2bfloat16_rn(mean - __bfloat162float(hi16));
+      } else {
+        vbar[o] = hi16;
+      }
     }
   }
 }
