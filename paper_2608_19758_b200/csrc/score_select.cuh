@@ -104,6 +104,7 @@ __device__ __forceinline__ void load_q_raw_async(uint8_t* sRaw, const uint8_t* _
                                                  const DevParams& P, int t, int nthr) {
   const int g = P.group;
   const uint32_t base = smem_u32(sRaw);
+  const uint64_t pol = l2_policy_evict_first();
   for (int i = t; i < kTileRows * 8; i += nthr) {
     const int row = i >> 3, ch = i & 7;
     const uint8_t* src = q;
@@ -115,7 +116,7 @@ __device__ __forceinline__ void load_q_raw_async(uint8_t* sRaw, const uint8_t* _
       src = q + (tok * P.num_q_heads + head) * kHeadDim + ch * 16;
       nbytes = 16;
     }
-    cp_async16(base + sw128_offset(row, ch), src, nbytes);
+    cp_async16(base + sw128_offset(row, ch), src, nbytes, pol);
   }
 }
 
@@ -173,6 +174,7 @@ __device__ __forceinline__ void load_q_tile_async(uint8_t* sQ, const uint8_t* __
                                                   const DevParams& P, int t, int nthr, bool wait = true) {
   const int g = P.group;
   const uint32_t base = smem_u32(sQ);
+  const uint64_t pol = l2_policy_evict_first();   // queries are read once
   for (int i = t; i < kTileRows * 16; i += nthr) {
     const int row = i >> 4, ch = i & 15;
     const uint8_t* src = q;
@@ -184,7 +186,7 @@ __device__ __forceinline__ void load_q_tile_async(uint8_t* sQ, const uint8_t* __
       src = q + ((tok * P.num_q_heads + head) * kHeadDim + ch * 8) * 2;
       nbytes = 16;
     }
-    cp_async16(base + (ch >> 3) * 16384 + sw128_offset(row, ch & 7), src, nbytes);
+    cp_async16(base + (ch >> 3) * 16384 + sw128_offset(row, ch & 7), src, nbytes, pol);
   }
   if (wait) cp_async_wait_all();
 }
@@ -297,6 +299,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
     if (lane == 0) {
       tma_prefetch_desc(&map_khi);
       tma_prefetch_desc(&map_klo);
+      const uint64_t keep = l2_policy_evict_last();
       uint32_t pc = 0;
       for (int it = 0;; ++it) {
         const int slot = it % kScoreInfoSlots;
@@ -312,8 +315,8 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
             uint8_t* dst = sStage + s * 32768;
             mbar_arrive_expect_tx(&full[s], 32768);
             const CUtensorMap* mp = part ? &map_klo : &map_khi;
-            tma_load_3d(dst, mp, &full[s], 0, h, blk_off + c * 128);
-            tma_load_3d(dst + 16384, mp, &full[s], 64, h, blk_off + c * 128);
+            tma_load_3d_hint(dst, mp, &full[s], 0, h, blk_off + c * 128, keep);
+            tma_load_3d_hint(dst + 16384, mp, &full[s], 64, h, blk_off + c * 128, keep);
           }
         }
         mbar_arrive(&info_empty[slot]);

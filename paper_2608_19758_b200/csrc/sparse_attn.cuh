@@ -362,6 +362,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     }
     uint32_t kc = 0, vc = 0, rc = 0;
     (void)rc;
+    const uint64_t keep = l2_policy_evict_last();   // K / V pages and pooled means: shared by many tiles
     const int ppb = P.pages_per_block, psz = P.page_size;
     for (int it = 0;; ++it) {
       const int slot = it & 1;
@@ -401,8 +402,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
               if (lane == 0) mbar_arrive_expect_tx(&raw_full[rs], rbytes);
               __syncwarp();
               if (pid >= 0)
-                tma_load_3d(sRaw + rs * kRawBytes + lane * psz * 128, kv ? &map_v : &map_k, &raw_full[rs], 0, sg.h,
-                            pid * psz);
+                tma_load_3d_hint(sRaw + rs * kRawBytes + lane * psz * 128, kv ? &map_v : &map_k, &raw_full[rs], 0, sg.h,
+                            pid * psz, keep);
             }
             ++kc;
             ++vc;
@@ -413,29 +414,29 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           if (lane == 0) mbar_arrive_expect_tx(&k_full[ks], bytes);
           __syncwarp();
           if (pid >= 0) {
-            tma_load_3d(dK + lane * psz * 128, &map_k, &k_full[ks], 0, sg.h, pid * psz);
-            tma_load_3d(dK + 16384 + lane * psz * 128, &map_k, &k_full[ks], 64, sg.h, pid * psz);
+            tma_load_3d_hint(dK + lane * psz * 128, &map_k, &k_full[ks], 0, sg.h, pid * psz, keep);
+            tma_load_3d_hint(dK + 16384 + lane * psz * 128, &map_k, &k_full[ks], 64, sg.h, pid * psz, keep);
           }
           if (vc >= kNV) mbar_wait(&v_empty[vs], ((vc / kNV) - 1) & 1, ctx, 303);
           if (lane == 0) mbar_arrive_expect_tx(&v_full[vs], bytes);
           __syncwarp();
           if (pid >= 0) {
-            tma_load_3d(dV + lane * psz * 128, &map_v, &v_full[vs], 0, sg.h, pid * psz);
-            tma_load_3d(dV + 16384 + lane * psz * 128, &map_v, &v_full[vs], 64, sg.h, pid * psz);
+            tma_load_3d_hint(dV + lane * psz * 128, &map_v, &v_full[vs], 0, sg.h, pid * psz, keep);
+            tma_load_3d_hint(dV + 16384 + lane * psz * 128, &map_v, &v_full[vs], 64, sg.h, pid * psz, keep);
           }
         } else {
           const int row0 = sg.blk_off + ti.chunk_id[i - T] * 128;
           if (kc >= kNK) mbar_wait(&k_empty[ks], ((kc / kNK) - 1) & 1, ctx, 304);
           if (lane == 0) {
             mbar_arrive_expect_tx(&k_full[ks], kTileBytes);
-            tma_load_3d(dK, &map_kbar, &k_full[ks], 0, sg.h, row0);
-            tma_load_3d(dK + 16384, &map_kbar, &k_full[ks], 64, sg.h, row0);
+            tma_load_3d_hint(dK, &map_kbar, &k_full[ks], 0, sg.h, row0, keep);
+            tma_load_3d_hint(dK + 16384, &map_kbar, &k_full[ks], 64, sg.h, row0, keep);
           }
           if (vc >= kNV) mbar_wait(&v_empty[vs], ((vc / kNV) - 1) & 1, ctx, 305);
           if (lane == 0) {
             mbar_arrive_expect_tx(&v_full[vs], kTileBytes);
-            tma_load_3d(dV, &map_vbar, &v_full[vs], 0, sg.h, row0);
-            tma_load_3d(dV + 16384, &map_vbar, &v_full[vs], 64, sg.h, row0);
+            tma_load_3d_hint(dV, &map_vbar, &v_full[vs], 0, sg.h, row0, keep);
+            tma_load_3d_hint(dV + 16384, &map_vbar, &v_full[vs], 64, sg.h, row0, keep);
           }
           __syncwarp();
         }
@@ -514,6 +515,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     const uint32_t o_addr = lane_base + 256 + wg * 64;   // this thread's 64 columns of O
     uint32_t sc0 = 0, sc1 = 0;   // completed uses of S0 / S1 (phases of s_full)
     uint32_t pv_base = 0;        // UMMA groups O += P V issued before this tile (phase of o_done)
+    const uint64_t stream_pol = l2_policy_evict_first();   // outputs are written once and not read here
     for (int it = 0;; ++it) {
       const int slot = it & 1;
       mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 501);
@@ -629,8 +631,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           o[j] = pack_bf16x2(v0, v1);
         }
         if (row_ok) {   // 32-byte stores: every instruction writes whole sectors
-          st_global_v8(orow + k * 32, &o[0]);
-          st_global_v8(orow + k * 32 + 16, &o[8]);
+          st_global_v8(orow + k * 32, &o[0], stream_pol);
+          st_global_v8(orow + k * 32 + 16, &o[8], stream_pol);
         }
       }
       if (wg == 0 && row_ok && A.lse != nullptr)
