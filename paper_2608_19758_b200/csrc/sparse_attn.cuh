@@ -20,9 +20,9 @@
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512).  P (BF16 pairs) has its own
 // columns, so S = Q K^T of iteration i+2 may start as soon as the softmax of iteration i has read S -- it does
-// not wait for O += P V of iteration i.  Issue order: QK(0) QK(1) PV(0) QK(2) PV(1) ...  Measured on B200:
-// consecutive UMMAs that differ in instruction descriptor or A source drain the pipe (~245 cycles), which
-// bounds this order at ~1510 cycles per 128x128 block against 1024 for back-to-back MMAs.
+// not wait for O += P V of iteration i.  Issue order: QK(0) QK(1) PV(0) QK(2) PV(1) ...  Per 128x128 block
+// the tensor pipe and the MUFU pipe are each busy 1024 cycles (ncu); how far the two overlap is what the
+// schedule decides.
 #pragma once
 #include <cuda_bf16.h>
 #include "common.cuh"
@@ -373,24 +373,28 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       const int T = ti.T, n_it = T + ti.nchunk;
       const int32_t* list = A.blk_idx + sg.off;
       const int32_t* pt = A.page_table + (size_t)sg.b * P.max_pages_per_seq;
+      // page id of this lane's page of exact iteration i (-1: past the end of the sequence, or not an exact
+      // iteration).  Fetched one iteration ahead: list entry -> page-table entry are two dependent global loads.
+      auto fetch_pid = [&](int i) -> int {
+        if (i >= T || lane >= ppb) return -1;
+        int J = ti.dense ? sg.J_hi - i : list[T - 1 - i];
+        J = max(0, min(J, sg.J_hi));
+        if (J * kBlock + lane * psz >= sg.Lk) return -1;
+        int pid = pt[J * ppb + lane];
+        if (pid < 0 || pid >= P.num_pages) {
+          atomicOr(A.status + ST_BAD_LIST, 2);
+          pid = -1;
+        }
+        return pid;
+      };
+      int pid_next = fetch_pid(0);
       for (int i = 0; i < n_it; ++i) {
         const int ks = kc % kNK, vs = vc % kNV;
         uint8_t* dK = sK + ks * kTileBytes;
         uint8_t* dV = sV + vs * kTileBytes;
+        const int pid = pid_next;
+        pid_next = fetch_pid(i + 1);
         if (i < T) {
-          int J = ti.dense ? sg.J_hi - i : list[T - 1 - i];
-          J = max(0, min(J, sg.J_hi));
-          int pid = -1;
-          if (lane < ppb) {
-            const int tok0 = J * kBlock + lane * psz;
-            if (tok0 < sg.Lk) {
-              pid = pt[J * ppb + lane];
-              if (pid < 0 || pid >= P.num_pages) {
-                atomicOr(A.status + ST_BAD_LIST, 2);
-                pid = -1;
-              }
-            }
-          }
           const int nvalid = __popc(__ballot_sync(0xffffffffu, pid >= 0));
           if constexpr (FP8) {
             // raw e4m3 tiles (128 bytes per token row) into the raw ring; the widening warpgroup fills the K / V rings
