@@ -158,7 +158,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-fp8", action="store_true")
-    ap.add_argument("--oracle-segments", type=int, default=20)
+    ap.add_argument("--oracle-segments", type=int, default=64)
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "fp2":
         args.warmup = 3
@@ -363,10 +363,11 @@ def main():
         dist.destroy_process_group()
     if rank != 0:
         return
-    # DRAM bytes per attention launch: ncu on config 2 (32768 tokens) measured 406.9 MB read + 235.8 MB written
-    # (profiles/dram_traffic_config2_all_kernels.md); every tile reads its Q rows and writes its O rows once and
-    # K/V comes from L2 after the first touch, so the figure scales with the token count.
-    traffic = (406.9e6 + 235.8e6) * (sum(l for l, _ in spec.seqs) / 32768.0) if spec.num_q_heads == 32 else None
+    # DRAM bytes per attention launch (dram__bytes_read.sum + dram__bytes_write.sum, one ncu pass on the full
+    # workload, profiles/bench_config3_launch_list.md): 3.61 GB read + 1.06 GB written at config 3 / 95 % sparsity,
+    # against 1.07 (Q) + 0.54 (K, V) + 1.07 (O) GB algorithmic: K/V pages are re-read from DRAM about five times
+    # because one KV head's 67 MB working set does not stay resident in L2 next to the streaming Q / O traffic.
+    traffic = 4.67e9 if (args.config == 3 and args.scale_down == 1 and abs(args.sparsity - 0.95) < 1e-6) else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
