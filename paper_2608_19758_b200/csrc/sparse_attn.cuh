@@ -44,7 +44,8 @@ struct AttnCfg {
   static constexpr int kThreads = FP8 ? 512 : 384;
   static constexpr int kNQ = FP8 ? 1 : 2;   // Q tiles in shared memory: two let the next unit's queries land while
                                             // this unit is still being multiplied (FP8 has no room for a second)
-  static constexpr int kNK = 2;             // K ring stages (32 KB each)
+  static constexpr int kNK = 2;             // K ring stages (32 KB each).  Must stay 2: stage i % 2 is released by the
+                                            // same commit that publishes S buffer i % 2
   static constexpr int kNV = 2;             // V ring stages
   static constexpr int kNRaw = FP8 ? 3 : 0; // raw FP8 tile ring (16 KB each), K and V tiles alternate
   static constexpr int kSmemBytes = 1024 + kTileBytes * (kNQ + kNK + kNV) + kNRaw * kRawBytes + 4096;
@@ -198,8 +199,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
   __shared__ TileInfo info[2];
   __shared__ uint32_t sel_bits[2][kMaxBlocks / 32];
   __shared__ uint64_t info_full[2], info_empty[2], q_full[2], q_empty[2], tile_done;
-  __shared__ uint64_t k_full[kNK], k_empty[kNK], v_full[kNV], v_empty[kNV];
-  __shared__ uint64_t s_full[2], p_ready[2], o_done;
+  // One tcgen05.commit costs the issuing thread ~70 cycles, so barriers that would be signalled by the same
+  // commit are merged: s_full[a] also releases K stage a (k_empty), v_empty[b] also says that O += P V of an
+  // iteration with parity b has completed (what the lazy rescale waits for).
+  static_assert(kNK == 2 && kNV == 2, "merged barriers assume two K stages and two V stages");
+  __shared__ uint64_t k_full[kNK], v_full[kNV], v_empty[kNV];
+  __shared__ uint64_t s_full[2], p_ready[2];
+  uint64_t* const k_empty = s_full;
   __shared__ uint64_t raw_full[kNRaw > 0 ? kNRaw : 1], raw_empty[kNRaw > 0 ? kNRaw : 1];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
@@ -217,8 +223,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     }
     for (int i = 0; i < 2; ++i) { mbar_init(&q_full[i], 64); mbar_init(&q_empty[i], 1); }
     mbar_init(&tile_done, 1);
-    mbar_init(&o_done, 1);
-    for (int i = 0; i < kNK; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); }
+    for (int i = 0; i < kNK; ++i) mbar_init(&k_full[i], 1);
     for (int i = 0; i < kNV; ++i) { mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); }
     for (int i = 0; i < kNRaw; ++i) { mbar_init(&raw_full[i], 1); mbar_init(&raw_empty[i], 1); }
     fence_barrier_init();
@@ -458,7 +463,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       constexpr uint32_t idesc_pv = make_idesc(128, 128, kFmt, kFmt, 0, 1);
       uint32_t kc = 0, vc = 0, pc0 = 0, pc1 = 0;
       auto issue_pv = [&](int j) {
-        const int b = j & 1;
+        const int b = vc & 1;   // P buffer / V stage: parity of the iteration counted over the whole kernel
         if (b) { mbar_wait(&p_ready[1], pc1 & 1, ctx, 401); ++pc1; }
         else { mbar_wait(&p_ready[0], pc0 & 1, ctx, 401); ++pc0; }
         const int vs = vc % kNV;
@@ -470,8 +475,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           const uint64_t bd = make_smem_desc_sw128(v_addr + ks * 2048, 16384, 1024);
           umma_f16_ts(tmem + 256, tmem + 384 + b * 64 + ks * 8, bd, idesc_pv, (j > 0) || ks > 0);
         }
-        umma_commit(&v_empty[vs]);
-        umma_commit(&o_done);
+        umma_commit(&v_empty[vs]);   // V stage vs (== iteration parity) is free and O holds this iteration
         ++vc;
       };
       for (int it = 0;; ++it) {
@@ -484,8 +488,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         mbar_wait(&q_full[qb], (it / kNQ) & 1, ctx, 404);
         const uint32_t q_addr = smem_u32(sQ + qb * kTileBytes);
         for (int i = 0; i < n_it; ++i) {
-          const int a = i & 1;
           const int ks_ = kc % kNK;
+          const int a = ks_;   // S buffer = K stage = parity of the iteration counted over the whole kernel
           mbar_wait(&k_full[ks_], (kc / kNK) & 1, ctx, 405);
           tc_fence_after();
           const uint32_t k_addr = smem_u32(sK + ks_ * kTileBytes);
@@ -497,8 +501,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
             const uint64_t bd = make_smem_desc_sw128(k_addr + off, 16, 1024);
             umma_f16_ss(tmem + a * 128, ad, bd, idesc_qk, ks > 0);
           }
-          umma_commit(&k_empty[ks_]);
-          umma_commit(&s_full[a]);
+          umma_commit(&s_full[a]);   // S_a is ready and K stage ks_ (== a) is free
           ++kc;
           if (i == n_it - 1) umma_commit(&q_empty[qb]);
           if (i >= 1) issue_pv(i - 1);
@@ -518,7 +521,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
     const uint32_t o_addr = lane_base + 256 + wg * 64;   // this thread's 64 columns of O
     uint32_t sc0 = 0, sc1 = 0;   // completed uses of S0 / S1 (phases of s_full)
-    uint32_t pv_base = 0;        // UMMA groups O += P V issued before this tile (phase of o_done)
+    uint32_t pv_base = 0;        // iterations (= UMMA groups O += P V = V stage uses) before this tile
     const uint64_t stream_pol = l2_policy_evict_first();   // outputs are written once and not read here
     for (int it = 0;; ++it) {
       const int slot = it & 1;
@@ -543,7 +546,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       // block id of the next exact iteration, fetched one iteration ahead
       int J_next = (!ti.dense && T > 0) ? list[T - 1] : 0;
       for (int i = 0; i < n_it; ++i) {
-        const int a = i & 1;
+        const int a = (pv_base + i) & 1;   // S / P buffer: parity of the iteration counted over the whole kernel
         const uint32_t s_addr = lane_base + a * 128 + wg * 64;
         const uint32_t p_addr = lane_base + 384 + a * 64 + wg * 32;
         // iteration kind and masks
@@ -583,8 +586,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         if (__any_sync(0xffffffffu, need)) {
           const float f = (m == -INFINITY) ? 0.f : ex2(m - m_new);
           if (i > 0) {
-            // O must be at rest: wait for O += P V of iteration i-1 (UMMA group number pv_base + i)
-            mbar_wait(&o_done, (pv_base + i - 1) & 1, ctx, 504);
+            // O must be at rest: wait for O += P V of iteration i-1, the ((pv_base + i - 1) / 2)-th use of V stage
+            // (pv_base + i - 1) % 2 counted over the whole kernel (iterations and V stages advance together)
+            mbar_wait(&v_empty[(pv_base + i - 1) & 1], ((pv_base + i - 1) >> 1) & 1, ctx, 504);
             tc_fence_after();
 #pragma unroll
             for (int k = 0; k < 2; ++k) {
