@@ -207,8 +207,8 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    if world > 1:                       # every rank an independent shard: same shape, its own seed
-        spec.config_id = spec.config_id * 10 + rank
+    from paper_2608_19758_b200 import shard
+    spec = shard.shard_spec(spec, rank, world)   # every rank an independent shard: same shape, its own seed
     case = inputs.make_case(spec)
     dc = binding.DeviceCase(case)
     peaks = measured_peaks()
@@ -284,11 +284,8 @@ def main():
     sel_pairs = float(dc.seg_count.sum().item())
     exec_flops = sel_pairs * 4.0 * 128 * 128 * 128
     ms_step = total_ms / args.steps
-    t = torch.tensor([ms_step], device="cuda", dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step_max = float(t.item())
-    value = world * dflops / (ms_step_max * 1e-3) / 1e12
+    value, ms_step_max, _ = shard.aggregate(dist, ms_step, dflops, device="cuda")
+    value /= 1e12
     att_mean = float(np.mean(att_ms))
     achieved = exec_flops / (att_mean * 1e-3) / 1e12
 
