@@ -246,6 +246,13 @@ static fp2_status set_attrs(fp2_plan* pl) {
       cudaFuncSetAttribute(sparse_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            AttnCfg<true>::kSmemBytes) != cudaSuccess)
     return FP2_ERR_CUDA;
+  // The attention kernels move registers between warps with setmaxnreg, whose wait is unbounded: launch only
+  // if the compiled kernels really own the registers the move assumes.
+  cudaFuncAttributes fa;
+  if (cudaFuncGetAttributes(&fa, sparse_attn_kernel<false>) != cudaSuccess) return FP2_ERR_CUDA;
+  if (fa.numRegs * AttnCfg<false>::kThreads < AttnCfg<false>::kRegsAfterMove) return FP2_ERR_UNSUPPORTED;
+  if (cudaFuncGetAttributes(&fa, sparse_attn_kernel<true>) != cudaSuccess) return FP2_ERR_CUDA;
+  if (fa.numRegs * AttnCfg<true>::kThreads < AttnCfg<true>::kRegsAfterMove) return FP2_ERR_UNSUPPORTED;
   pl->attrs_set = true;
   return FP2_OK;
 }

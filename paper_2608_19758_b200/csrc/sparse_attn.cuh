@@ -8,15 +8,16 @@
 // a correction chunk stages 128 consecutive pooled (kbar, vbar) rows exactly like a KV block, its logits are
 // shifted by log2(128) (every corrected block is full) and masked by todo = fully-visible & ~selected.
 //
-// Roles (12 warps):
-//   warps 0-7  two softmax warpgroups.  Both work on EVERY iteration: warpgroup w owns logit columns
-//              [64w, 64w+64) of all 128 rows (thread = row).  They exchange the row maximum through shared
-//              memory once per iteration, so the softmax latency of a block is halved and one accumulator O
-//              serves the whole tile (no merge at the end).
-//   warp 8     TMA producer: K / V pages through the page table into two rings (Eq. 22)
-//   warp 9     UMMA issuer: S = Q K^T (SS), O += P V (P read from TMEM, V MN-major from shared memory)
-//   warps 10-11 tile set-up: fetch the next unit, validate its list, build the correction masks, stage Q
-//   warps 12-15 (FP8 inputs only) widen raw e4m3 K / V tiles to F16 into the K / V rings
+// Roles:
+//   warps 0..4W-1   W = kWG softmax warpgroups (2 by default).  All work on EVERY iteration: warpgroup w owns
+//              logit columns [w 128/W, (w+1) 128/W) of all 128 rows (thread = row).  They exchange the row maximum
+//              through shared memory once per iteration; one accumulator O serves the whole tile (no merge at the
+//              end).  W = 4 (four warps per scheduler, 104 registers each) builds and passes parity but measured
+//              3 % (dense) to 10 % (sparse) slower at 32K than W = 2 with 224 registers.
+//   warp 4W    TMA producer: K / V pages through the page table into two rings (Eq. 22)
+//   warp 4W+1  UMMA issuer: S = Q K^T (SS), O += P V (P read from TMEM, V MN-major from shared memory)
+//   warps 4W+2, 4W+3  tile set-up: fetch the next unit, validate its list, build the correction masks, stage Q
+//   warps 4W+4..4W+7  (FP8 inputs only) widen raw e4m3 K / V tiles to F16 into the K / V rings
 //
 // TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512).  P (BF16 pairs) has its own
 // columns, so S = Q K^T of iteration i+2 may start as soon as the softmax of iteration i has read S -- it does
@@ -39,16 +40,34 @@ constexpr int kRawBytes = 16384;    // one 128 x 128 tile of FP8 elements as TMA
 // with F16 operands (Q widened when staged, P packed as F16).  The per-head scales never touch the operands:
 // q_scale * k_scale multiplies the logits of a row, v_scale multiplies the output.  A single e4m3 probability
 // tile, the other way to feed FP8 V to the tensor core, costs ~0.06 max-abs output error by itself.
+#ifndef FP2_SOFTMAX_WGS
+#define FP2_SOFTMAX_WGS 2
+#endif
+constexpr int kWG = FP2_SOFTMAX_WGS;      // softmax warpgroups; each owns 128 / kWG logit columns of every row
+constexpr int kCW = 128 / kWG;            // columns per warpgroup (64 or 32)
+constexpr int kSW = 4 * kWG;              // softmax warps; the service warps follow them
+static_assert(kWG == 2 || kWG == 4, "two or four softmax warpgroups");
+
 template <bool FP8>
 struct AttnCfg {
-  static constexpr int kThreads = FP8 ? 512 : 384;
+  static constexpr int kThreads = 128 * kWG + 128 + (FP8 ? 128 : 0);
   static constexpr int kNQ = FP8 ? 1 : 2;   // Q tiles in shared memory: two let the next unit's queries land while
                                             // this unit is still being multiplied (FP8 has no room for a second)
   static constexpr int kNK = 2;             // K ring stages (32 KB each).  Must stay 2: stage i % 2 is released by the
                                             // same commit that publishes S buffer i % 2
   static constexpr int kNV = 2;             // V ring stages
   static constexpr int kNRaw = FP8 ? 3 : 0; // raw FP8 tile ring (16 KB each), K and V tiles alternate
-  static constexpr int kSmemBytes = 1024 + kTileBytes * (kNQ + kNK + kNV) + kNRaw * kRawBytes + 4096;
+  static constexpr int kSmemBytes = 1024 + kTileBytes * (kNQ + kNK + kNV) + kNRaw * kRawBytes + 2048 * kWG;
+  // Registers.  The CTA is launched with kRegsBase registers per thread (what __launch_bounds__(kThreads, 1)
+  // lets ptxas use); setmaxnreg then moves registers from the service warps (kRegsService) to the softmax warps
+  // (kRegsSoftmax).  setmaxnreg.inc waits -- without bound -- until the CTA's own pool has the registers, so the
+  // total after the move must not exceed the launch allocation; the host checks the compiled register count
+  // against kRegsAfterMove before the first launch and refuses to launch otherwise.
+  static constexpr int kRegsBase = (65536 / kThreads) / 8 * 8;
+  static constexpr int kRegsService = (kWG == 4) ? 48 : 56;
+  static constexpr int kRegsSoftmax = (kWG == 4) ? (FP8 ? 96 : 104) : (FP8 ? 200 : 224);
+  static constexpr int kRegsAfterMove = (kThreads - 128 * kWG) * kRegsService + 128 * kWG * kRegsSoftmax;
+  static_assert(kRegsAfterMove <= kThreads * kRegsBase, "register budget: setmaxnreg.inc would wait forever");
   static constexpr int kFmt = FP8 ? 0 : 1;  // UMMA kind::f16 operand format: 0 = F16, 1 = BF16
 };
 
@@ -80,20 +99,19 @@ struct AttnArgs {
 
 // Masked iterations (diagonal blocks, correction chunks -- the minority): overwrite the hidden logits of this
 // thread's row with -inf in TMEM, so that the softmax step itself carries no mask logic (predicating the mask
-// into the softmax body cost 2.5x on every iteration, masked or not).  The thread owns 64 columns starting at
-// block column col0; column j stays visible iff j <= tok_lim and bit (j - col0) of {cm_lo, cm_hi} is set.
-__device__ __forceinline__ void mask_half(uint32_t s_addr, int col0, int tok_lim, uint32_t cm_lo, uint32_t cm_hi) {
+// into the softmax body cost 2.5x on every iteration, masked or not).  The thread owns kCW columns starting at
+// block column col0; column j stays visible iff j <= tok_lim and bit (j - col0) of cm (32 bits per word) is set.
+__device__ __forceinline__ void mask_cols(uint32_t s_addr, int col0, int tok_lim, const uint32_t* cm) {
 #pragma unroll
-  for (int k = 0; k < 2; ++k) {
-    const uint32_t cm = k ? cm_hi : cm_lo;
-    const bool all_vis = (col0 + k * 32 + 31 <= tok_lim) && (cm == 0xffffffffu);
+  for (int k = 0; k < kCW / 32; ++k) {
+    const bool all_vis = (col0 + k * 32 + 31 <= tok_lim) && (cm[k] == 0xffffffffu);
     if (__all_sync(0xffffffffu, all_vis)) continue;   // TMEM accesses are warp-wide: decide per warp
     uint32_t rr[32];
     tmem_ld32(s_addr + k * 32, rr);
     tmem_wait_ld();
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
-      const bool vis = (col0 + k * 32 + j <= tok_lim) && ((cm >> j) & 1u);
+      const bool vis = (col0 + k * 32 + j <= tok_lim) && ((cm[k] >> j) & 1u);
       rr[j] = vis ? rr[j] : 0xff800000u;  // -inf
     }
     tmem_st32(s_addr + k * 32, rr);
@@ -101,35 +119,37 @@ __device__ __forceinline__ void mask_half(uint32_t s_addr, int col0, int tok_lim
   tmem_wait_st();
 }
 
-// Row maximum of this thread's 64 logit columns (raw, unscaled): two TMEM loads in flight, eight chains of
+// Row maximum of this thread's kCW logit columns (raw, unscaled): all TMEM loads in flight, chains of
 // three-input maxima.
-__device__ __forceinline__ float half_row_max(uint32_t s_addr) {
-  uint32_t sv[64];
-  tmem_ld32(s_addr, reinterpret_cast<uint32_t(&)[32]>(sv[0]));
-  tmem_ld32(s_addr + 32, reinterpret_cast<uint32_t(&)[32]>(sv[32]));
-  tmem_wait_ld();
-  float mx8[8];
+__device__ __forceinline__ float cols_row_max(uint32_t s_addr) {
+  uint32_t sv[kCW];
 #pragma unroll
-  for (int c = 0; c < 8; ++c) {
+  for (int k = 0; k < kCW / 32; ++k) tmem_ld32(s_addr + k * 32, reinterpret_cast<uint32_t(&)[32]>(sv[k * 32]));
+  tmem_wait_ld();
+  float mx8[kCW / 8];
+#pragma unroll
+  for (int c = 0; c < kCW / 8; ++c) {
     const float* v = reinterpret_cast<const float*>(&sv[c * 8]);
     mx8[c] = fmaxf(max3(max3(v[0], v[1], v[2]), v[3], v[4]), max3(v[5], v[6], v[7]));
   }
-  return fmaxf(max3(mx8[0], mx8[1], mx8[2]), max3(max3(mx8[3], mx8[4], mx8[5]), mx8[6], mx8[7]));
+  float r = fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3]));
+  if constexpr (kCW == 64) r = fmaxf(r, fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
+  return r;
 }
 
-// p = 2^(s * cs + neg_m) for this thread's 64 columns, written as 16-bit pairs to 32 columns at p_addr.
-// The second TMEM load is in flight while the first half is exponentiated.  Scaling and row sum use packed
-// fp32x2 instructions.  Returns the row's partial sum.
+// p = 2^(s * cs + neg_m) for this thread's kCW columns, written as 16-bit pairs to kCW / 2 columns at p_addr.
+// With two 32-column chunks the second TMEM load is in flight while the first chunk is exponentiated.  Scaling
+// and row sum use packed fp32x2 instructions.  Returns the row's partial sum.
 template <bool F16>
-__device__ __forceinline__ float half_row_exp(uint32_t s_addr, uint32_t p_addr, float cs, float neg_m) {
+__device__ __forceinline__ float cols_row_exp(uint32_t s_addr, uint32_t p_addr, float cs, float neg_m) {
   const uint64_t cs2 = f2_pack(cs, cs), nm2 = f2_pack(neg_m, neg_m);
   uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};   // four independent (lo, hi) accumulators, +0.0f bit patterns
-  uint32_t buf[2][32];
+  uint32_t buf[kCW / 32][32];
   tmem_ld32(s_addr, buf[0]);
   tmem_wait_ld();
 #pragma unroll
-  for (int k = 0; k < 2; ++k) {
-    if (k == 0) tmem_ld32(s_addr + 32, buf[1]);
+  for (int k = 0; k < kCW / 32; ++k) {
+    if (k + 1 < kCW / 32) tmem_ld32(s_addr + (k + 1) * 32, buf[(k + 1) % (kCW / 32)]);
     uint32_t pk[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
@@ -140,12 +160,11 @@ __device__ __forceinline__ float half_row_exp(uint32_t s_addr, uint32_t p_addr, 
       sum2[j & 3] = f2_add(sum2[j & 3], f2_pack(p0, p1));
       pk[j] = F16 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1);
     }
-    if (k == 0) tmem_wait_ld();
+    if (k + 1 < kCW / 32) tmem_wait_ld();
     tmem_st16(p_addr + k * 16, pk);
   }
-  float a0, a1, b0, b1;
+  float a0, a1;
   f2_unpack(f2_add(f2_add(sum2[0], sum2[1]), f2_add(sum2[2], sum2[3])), a0, a1);
-  (void)b0; (void)b1;
   return a0 + a1;
 }
 
@@ -194,7 +213,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
   uint8_t* sK = smem + kNQ * kTileBytes;
   uint8_t* sV = sK + kNK * kTileBytes;
   uint8_t* sRaw = sV + kNV * kTileBytes;                          // FP8 only: raw tile ring
-  float* sX = reinterpret_cast<float*>(sRaw + kNRaw * kRawBytes);  // [2 parity][2 wg][128] row-max / row-sum exchange
+  float* sX = reinterpret_cast<float*>(sRaw + kNRaw * kRawBytes);  // [2 parity][kWG][128] row-max exchange, then the same for row sums
 
   __shared__ TileInfo info[2];
   __shared__ uint32_t sel_bits[2][kMaxBlocks / 32];
@@ -217,9 +236,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     abort_flag = 0;
     for (int i = 0; i < 2; ++i) {
       mbar_init(&info_full[i], 1);
-      mbar_init(&info_empty[i], 2 + 256 + (FP8 ? 1 : 0));
+      mbar_init(&info_empty[i], 2 + 128 * kWG + (FP8 ? 1 : 0));
       mbar_init(&s_full[i], 1);
-      mbar_init(&p_ready[i], 256);
+      mbar_init(&p_ready[i], 128 * kWG);
     }
     for (int i = 0; i < 2; ++i) { mbar_init(&q_full[i], 64); mbar_init(&q_empty[i], 1); }
     mbar_init(&tile_done, 1);
@@ -232,7 +251,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
   // there is multiplied by probabilities that are exactly zero, so it must be finite.
   for (int i = tid; i < ((kNK + kNV) * kTileBytes + kNRaw * kRawBytes) / 16; i += kAttnThreads)
     reinterpret_cast<uint4*>(sK)[i] = make_uint4(0, 0, 0, 0);
-  if (warp == 9) {
+  if (warp == kSW + 1) {
     tmem_alloc(&tmem_base_s, 512);
     tmem_relinquish();
   }
@@ -243,11 +262,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
   const uint32_t tmem = tmem_base_s;
   const int g = P.group;
 
-  if (FP8 && warp >= 12) {
+  if (FP8 && warp >= kSW + 4) {
     // =============================== FP8 -> F16 widening warpgroup ===============================
-    setmaxnreg_dec<56>();
+    setmaxnreg_dec<AttnCfg<FP8>::kRegsService>();
     if constexpr (FP8) {
-      const int t128 = tid - 384;
+      const int t128 = tid - 32 * (kSW + 4);
       uint32_t kc = 0, vc = 0, rc = 0;
       for (int it = 0;; ++it) {
         const int slot = it & 1;
@@ -279,10 +298,10 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         if (t128 == 0) mbar_arrive(&info_empty[slot]);
       }
     }
-  } else if (warp >= 10) {
+  } else if (warp >= kSW + 2) {
     // =============================== tile set-up + Q staging ===============================
-    setmaxnreg_dec<56>();
-    const int t64 = tid - 320;
+    setmaxnreg_dec<AttnCfg<FP8>::kRegsService>();
+    const int t64 = tid - 32 * (kSW + 2);
     for (int it = 0;; ++it) {
       const int slot = it & 1;
       if (it >= 2) mbar_wait(&info_empty[slot], ((it >> 1) - 1) & 1, ctx, 201);
@@ -356,9 +375,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       fence_proxy_async();
       mbar_arrive(&q_full[qb]);
     }
-  } else if (warp == 8) {
+  } else if (warp == kSW) {
     // =============================== TMA producer ===============================
-    setmaxnreg_dec<56>();
+    setmaxnreg_dec<AttnCfg<FP8>::kRegsService>();
     if (lane == 0) {
       tma_prefetch_desc(&map_k);
       tma_prefetch_desc(&map_v);
@@ -454,9 +473,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       }
       if (lane == 0) mbar_arrive(&info_empty[slot]);
     }
-  } else if (warp == 9) {
+  } else if (warp == kSW + 1) {
     // =============================== UMMA issuer ===============================
-    setmaxnreg_dec<56>();
+    setmaxnreg_dec<AttnCfg<FP8>::kRegsService>();
     if (lane == 0) {
       constexpr int kFmt = AttnCfg<FP8>::kFmt;
       constexpr uint32_t idesc_qk = make_idesc(128, 128, kFmt, kFmt, 0, 0);
@@ -514,12 +533,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     }
   } else {
     // =============================== softmax warpgroups + epilogue ===============================
-    // register budget: 384 threads: 128 x 56 + 256 x 224 = 64512; 512 threads (FP8): 256 x 56 + 256 x 200 = 65536
-    setmaxnreg_inc<FP8 ? 200 : 224>();
+    setmaxnreg_inc<AttnCfg<FP8>::kRegsSoftmax>();
     const int wg = warp >> 2;
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    const uint32_t o_addr = lane_base + 256 + wg * 64;   // this thread's 64 columns of O
+    const uint32_t o_addr = lane_base + 256 + wg * kCW;   // this thread's kCW columns of O
     uint32_t sc0 = 0, sc1 = 0;   // completed uses of S0 / S1 (phases of s_full)
     uint32_t pv_base = 0;        // iterations (= UMMA groups O += P V = V stage uses) before this tile
     const uint64_t stream_pol = l2_policy_evict_first();   // outputs are written once and not read here
@@ -547,12 +565,14 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       int J_next = (!ti.dense && T > 0) ? list[T - 1] : 0;
       for (int i = 0; i < n_it; ++i) {
         const int a = (pv_base + i) & 1;   // S / P buffer: parity of the iteration counted over the whole kernel
-        const uint32_t s_addr = lane_base + a * 128 + wg * 64;
-        const uint32_t p_addr = lane_base + 384 + a * 64 + wg * 32;
+        const uint32_t s_addr = lane_base + a * 128 + wg * kCW;
+        const uint32_t p_addr = lane_base + 384 + a * 64 + wg * (kCW / 2);
         // iteration kind and masks
         bool need_mask = false;
         int tok_lim = 1 << 30;     // exact block: columns j with j <= tok_lim are visible
-        uint32_t cm_lo = 0xffffffffu, cm_hi = 0xffffffffu;
+        uint32_t cm[kCW / 32];
+#pragma unroll
+        for (int w = 0; w < kCW / 32; ++w) cm[w] = 0xffffffffu;
         float shift = 0.f, cs = cs_exact;
         if (i < T) {
           int J = ti.dense ? sg.J_hi - i : J_next;
@@ -562,8 +582,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           tok_lim = pos - J * kBlock;
         } else {
           const int c = ti.chunk_id[i - T];
-          cm_lo = ti.todo[c][2 * wg];
-          cm_hi = ti.todo[c][2 * wg + 1];
+#pragma unroll
+          for (int w = 0; w < kCW / 32; ++w) cm[w] = ti.todo[c][wg * (kCW / 32) + w];
           shift = 7.0f;  // log2(128): one pooled row stands for a full block (Eq. 6)
           cs = cs_chunk;
           need_mask = true;
@@ -571,13 +591,14 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         if (a) { mbar_wait(&s_full[1], sc1 & 1, ctx, 502); ++sc1; }
         else { mbar_wait(&s_full[0], sc0 & 1, ctx, 502); ++sc0; }
         tc_fence_after();
-        if (need_mask) mask_half(s_addr, wg * 64, tok_lim, cm_lo, cm_hi);
+        if (need_mask) mask_cols(s_addr, wg * kCW, tok_lim, cm);
         // row maximum over all 128 columns: own half, then the other warpgroup's through shared memory
-        float mx = half_row_max(s_addr);
-        float* xch = sX + (i & 1) * 256;
+        float mx = cols_row_max(s_addr);
+        float* xch = sX + (i & 1) * (kWG * 128);
         xch[wg * 128 + row] = mx;
-        named_bar_sync(1, 256);
-        mx = fmaxf(mx, xch[(wg ^ 1) * 128 + row]);
+        named_bar_sync(1, 128 * kWG);
+#pragma unroll
+        for (int w = 1; w < kWG; ++w) mx = fmaxf(mx, xch[((wg + w) % kWG) * 128 + row]);
         mx = fmaf(mx, cs, shift);  // cs > 0: scaling commutes with the maximum
         const float m_new = fmaxf(m, mx);
         // lazy rescale: only when some row of the warp moved its maximum by more than 2^8.  Both warpgroups
@@ -591,7 +612,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
             mbar_wait(&v_empty[(pv_base + i - 1) & 1], ((pv_base + i - 1) >> 1) & 1, ctx, 504);
             tc_fence_after();
 #pragma unroll
-            for (int k = 0; k < 2; ++k) {
+            for (int k = 0; k < kCW / 32; ++k) {
               uint32_t rr[32];
               tmem_ld32(o_addr + k * 32, rr);
               tmem_wait_ld();
@@ -605,7 +626,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         }
         // a row with nothing visible so far has m = -inf and only -inf logits: exponent against 0 -> zeros
         const float neg_m = (m == -INFINITY) ? shift : shift - m;
-        l += half_row_exp<FP8>(s_addr, p_addr, cs, neg_m);
+        l += cols_row_exp<FP8>(s_addr, p_addr, cs, neg_m);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&p_ready[a]);
@@ -614,18 +635,20 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       // ------------------------------ epilogue ------------------------------
       mbar_wait(&tile_done, it & 1, ctx, 503);
       tc_fence_after();
-      float* xch = sX + 512 + (it & 1) * 256;   // by tile parity: no barrier is needed before its next use
+      float* xch = sX + 2 * kWG * 128 + (it & 1) * (kWG * 128);   // by tile parity: no barrier before its next use
       xch[wg * 128 + row] = l;
-      named_bar_sync(1, 256);
-      const float L = l + xch[(wg ^ 1) * 128 + row];
+      named_bar_sync(1, 128 * kWG);
+      float L = l;
+#pragma unroll
+      for (int w = 1; w < kWG; ++w) L += xch[((wg + w) % kWG) * 128 + row];
       const float inv = L > 0.f ? out_scale / L : 0.f;
       const bool have_o = n_it >= 1;
       const bool row_ok = row < sg.nrows;
       const size_t tok = (size_t)sg.q_tok0 + r / g;
       const int head = sg.h * g + r % g;
-      __nv_bfloat16* orow = A.out + (tok * P.num_q_heads + head) * kHeadDim + wg * 64;
+      __nv_bfloat16* orow = A.out + (tok * P.num_q_heads + head) * kHeadDim + wg * kCW;
 #pragma unroll
-      for (int k = 0; k < 2; ++k) {
+      for (int k = 0; k < kCW / 32; ++k) {
         uint32_t a0[32];
         if (have_o) {
           tmem_ld32(o_addr + k * 32, a0);
@@ -653,7 +676,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
   if (abort_flag) __nanosleep(2000000);
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) tmem_dealloc(tmem, 512);
+  if (warp == kSW + 1) tmem_dealloc(tmem, 512);
 }
 
 }  // namespace fp2
