@@ -119,10 +119,9 @@ __device__ __forceinline__ void mask_cols(uint32_t s_addr, int col0, int tok_lim
   tmem_wait_st();
 }
 
-// Row maximum of this thread's kCW logit columns (raw, unscaled): all TMEM loads in flight, chains of
-// three-input maxima.
-__device__ __forceinline__ float cols_row_max(uint32_t s_addr) {
-  uint32_t sv[kCW];
+// This thread's kCW logit columns (raw, unscaled) into registers, and their maximum: all TMEM loads in flight,
+// chains of three-input maxima.
+__device__ __forceinline__ float cols_row_max(uint32_t s_addr, uint32_t (&sv)[kCW]) {
 #pragma unroll
   for (int k = 0; k < kCW / 32; ++k) tmem_ld32(s_addr + k * 32, reinterpret_cast<uint32_t(&)[32]>(sv[k * 32]));
   tmem_wait_ld();
@@ -137,30 +136,27 @@ __device__ __forceinline__ float cols_row_max(uint32_t s_addr) {
   return r;
 }
 
-// p = 2^(s * cs + neg_m) for this thread's kCW columns, written as 16-bit pairs to kCW / 2 columns at p_addr.
-// With two 32-column chunks the second TMEM load is in flight while the first chunk is exponentiated.  Scaling
-// and row sum use packed fp32x2 instructions.  Returns the row's partial sum.
+// p = 2^(s * cs + neg_m) for this thread's kCW logits (still in the registers the maximum pass loaded them into),
+// written as 16-bit pairs to kCW / 2 columns at p_addr.  One TMEM read per logit: besides the latency, TMEM
+// loads of the softmax warps lengthen the time the tensor pipe takes to accept each MMA of the issuing thread.
+// Scaling and row sum use packed fp32x2 instructions.  Returns the row's partial sum.
 template <bool F16>
-__device__ __forceinline__ float cols_row_exp(uint32_t s_addr, uint32_t p_addr, float cs, float neg_m) {
+__device__ __forceinline__ float cols_row_exp(const uint32_t (&sv)[kCW], uint32_t p_addr, float cs, float neg_m) {
   const uint64_t cs2 = f2_pack(cs, cs), nm2 = f2_pack(neg_m, neg_m);
   uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};   // four independent (lo, hi) accumulators, +0.0f bit patterns
-  uint32_t buf[kCW / 32][32];
-  tmem_ld32(s_addr, buf[0]);
-  tmem_wait_ld();
 #pragma unroll
   for (int k = 0; k < kCW / 32; ++k) {
-    if (k + 1 < kCW / 32) tmem_ld32(s_addr + (k + 1) * 32, buf[(k + 1) % (kCW / 32)]);
     uint32_t pk[16];
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
-      const uint64_t x2 = f2_fma(f2_pack(__uint_as_float(buf[k][2 * j]), __uint_as_float(buf[k][2 * j + 1])), cs2, nm2);
+      const uint64_t x2 =
+          f2_fma(f2_pack(__uint_as_float(sv[k * 32 + 2 * j]), __uint_as_float(sv[k * 32 + 2 * j + 1])), cs2, nm2);
       float x0, x1;
       f2_unpack(x2, x0, x1);
       const float p0 = ex2(x0), p1 = ex2(x1);
       sum2[j & 3] = f2_add(sum2[j & 3], f2_pack(p0, p1));
       pk[j] = F16 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1);
     }
-    if (k + 1 < kCW / 32) tmem_wait_ld();
     tmem_st16(p_addr + k * 16, pk);
   }
   float a0, a1;
@@ -593,7 +589,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         tc_fence_after();
         if (need_mask) mask_cols(s_addr, wg * kCW, tok_lim, cm);
         // row maximum over all 128 columns: own half, then the other warpgroup's through shared memory
-        float mx = cols_row_max(s_addr);
+        uint32_t sv[kCW];
+        float mx = cols_row_max(s_addr, sv);
         float* xch = sX + (i & 1) * (kWG * 128);
         xch[wg * 128 + row] = mx;
         named_bar_sync(1, 128 * kWG);
@@ -626,7 +623,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         }
         // a row with nothing visible so far has m = -inf and only -inf logits: exponent against 0 -> zeros
         const float neg_m = (m == -INFINITY) ? shift : shift - m;
-        l += cols_row_exp<FP8>(s_addr, p_addr, cs, neg_m);
+        l += cols_row_exp<FP8>(sv, p_addr, cs, neg_m);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&p_ready[a]);
