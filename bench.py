@@ -372,7 +372,7 @@ def main():
         "config": {"workload": workload, "target_sparsity": args.sparsity, "l2": "inputs (Q 1.07 GB, K+V 0.54 GB) "
                    "exceed the 126 MB L2; no flush", "step": "fp2_select_blocks + fp2_sparse_prefill"},
         "clocks": clocks, "gpu_launches": launches,
-        "roofline": {"bound": "tensor", "kernel": "sparse_attn_kernel", "achieved": achieved,
+        "roofline": {"bound": "tensor", "kernel": "sparse_attn_bf16_kernel", "achieved": achieved,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
                      "peak_source": peaks["source"] + " burst bf16 GEMM", "traffic": traffic,
                      "flops_per_launch": exec_flops, "ms_per_launch": att_mean,

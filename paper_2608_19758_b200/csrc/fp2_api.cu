@@ -14,6 +14,7 @@
 #include "pool_kv.cuh"
 #include "score_select.cuh"
 #include "sparse_attn.cuh"
+#include "sparse_attn_bf16.cuh"
 
 using namespace fp2;
 
@@ -241,16 +242,16 @@ static fp2_status set_attrs(fp2_plan* pl) {
                            kScoreSmemBytes) != cudaSuccess ||
       cudaFuncSetAttribute(score_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kScoreSmemBytes) != cudaSuccess ||
-      cudaFuncSetAttribute(sparse_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           AttnCfg<false>::kSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(sparse_attn_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           AttnBf16Cfg::kSmemBytes) != cudaSuccess ||
       cudaFuncSetAttribute(sparse_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            AttnCfg<true>::kSmemBytes) != cudaSuccess)
     return FP2_ERR_CUDA;
   // The attention kernels move registers between warps with setmaxnreg, whose wait is unbounded: launch only
   // if the compiled kernels really own the registers the move assumes.
   cudaFuncAttributes fa;
-  if (cudaFuncGetAttributes(&fa, sparse_attn_kernel<false>) != cudaSuccess) return FP2_ERR_CUDA;
-  if (fa.numRegs * AttnCfg<false>::kThreads < AttnCfg<false>::kRegsAfterMove) return FP2_ERR_UNSUPPORTED;
+  if (cudaFuncGetAttributes(&fa, sparse_attn_bf16_kernel) != cudaSuccess) return FP2_ERR_CUDA;
+  if (fa.numRegs * AttnBf16Cfg::kThreads < AttnBf16Cfg::kRegsAfterMove) return FP2_ERR_UNSUPPORTED;
   if (cudaFuncGetAttributes(&fa, sparse_attn_kernel<true>) != cudaSuccess) return FP2_ERR_CUDA;
   if (fa.numRegs * AttnCfg<true>::kThreads < AttnCfg<true>::kRegsAfterMove) return FP2_ERR_UNSUPPORTED;
   pl->attrs_set = true;
@@ -339,6 +340,14 @@ extern "C" fp2_status fp2_select_blocks(fp2_plan* pl, const void* q, const void*
 // ------------------------------------------------------------------------------------------------------
 // stage 2 (sparse and dense)
 // ------------------------------------------------------------------------------------------------------
+// BF16 attention: two 256-thread CTAs per SM, each a persistent worker on the shared work counter.
+static void launch_attn_bf16(fp2_plan* pl, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mkb,
+                             const CUtensorMap& mvb, const AttnArgs& a, cudaStream_t st) {
+  const int64_t workers = (int64_t)pl->num_sms * AttnBf16Cfg::kCtasPerSm;
+  const unsigned grid = (unsigned)(pl->nseg < workers ? pl->nseg : workers);
+  sparse_attn_bf16_kernel<<<grid, AttnBf16Cfg::kThreads, AttnBf16Cfg::kSmemBytes, st>>>(mk, mv, mkb, mvb, a, pl->dev);
+}
+
 static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, const void* v, const int32_t* pt,
                                 const int32_t* cu, const int32_t* lk, const int32_t* seg_count,
                                 const int32_t* blk_idx, const float* qs, const float* ks, const float* vs, void* out,
@@ -377,8 +386,7 @@ static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, cons
     sparse_attn_kernel<true><<<grid, AttnCfg<true>::kThreads, AttnCfg<true>::kSmemBytes, st>>>(mk, mv, mkb, mvb, a,
                                                                                               pl->dev);
   else
-    sparse_attn_kernel<false><<<grid, AttnCfg<false>::kThreads, AttnCfg<false>::kSmemBytes, st>>>(mk, mv, mkb, mvb,
-                                                                                                 a, pl->dev);
+    launch_attn_bf16(pl, mk, mv, mkb, mvb, a, st);
   pl->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
@@ -475,10 +483,8 @@ extern "C" fp2_status fp2_dense_prefill_static(fp2_plan* pl, const void* q, cons
   a.lse = lse;
   a.work_counter = reinterpret_cast<int*>(sw + 64);
   a.status = reinterpret_cast<int*>(sw);
-  const unsigned grid = (unsigned)(pl->nseg < pl->num_sms ? pl->nseg : pl->num_sms);
   // the dense path stages no pooled chunks: the two pooled-mean maps are never dereferenced
-  sparse_attn_kernel<false><<<grid, AttnCfg<false>::kThreads, AttnCfg<false>::kSmemBytes, st>>>(mk, mv, mk, mv, a,
-                                                                                               pl->dev);
+  launch_attn_bf16(pl, mk, mv, mk, mv, a, st);
   pl->last_launches = 4;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }

@@ -1,0 +1,510 @@
+// Block-sparse causal flash attention with mean correction (Eq. 4, Eq. 6; Algorithm 1 lines 6-11) for BF16
+// inputs: the same computation, work units, lists and outputs as sparse_attn_kernel, laid out as TWO small
+// CTAs per SM instead of one large one.
+//
+// Per 128x128 block the tensor pipe (two GEMMs) and the MUFU pipe (16384 exponentials) are each busy 1024
+// cycles, and a softmax step has several hundred cycles of latency around its exponentials (TMEM load, row
+// maximum, TMEM store, barrier hand-overs).  Two warpgroups that share one tile must exchange row maxima and so
+// move in lockstep: both are in their latency phase at the same time and the MUFU pipe idles.  Here every CTA
+// has ONE softmax warpgroup that owns whole rows (thread = row, 128 logits in registers), nothing crosses
+// between the two CTAs of an SM, and they drift out of phase by themselves: while one CTA's warps stream
+// exponentials the other's wait for the tensor pipe, load logits or hand over P.
+//
+// One CTA: 256 threads, 96 KB of tile memory (Q, one K stage, one V stage), 256 TMEM columns:
+//   S [0,128)  logits of the iteration; P (BF16 pairs) overwrites its first 64 columns in place
+//   O [128,256)
+// Everything is single-buffered: S = Q K^T of iteration i+1 is issued behind O += P V of iteration i (which
+// reads P out of the S columns), the K tile of i+1 is requested when S = Q K^T (i) has completed and the V tile
+// when O += P V (i) has.  The other CTA of the SM fills the bubbles this leaves.
+//
+// Roles: warps 0..3 softmax + epilogue; warp 4 TMA producer (Eq. 22); warp 5 UMMA issuer (and TMEM owner);
+// warps 6, 7 unit set-up (fetch the next unit, validate its list, build the correction masks, stage Q).
+#pragma once
+#include <cuda_bf16.h>
+#include "common.cuh"
+#include "ptx.cuh"
+#include "score_select.cuh"  // load_q_tile_async
+#include "sparse_attn.cuh"   // TileInfo, AttnArgs, kTileBytes
+
+namespace fp2 {
+
+struct AttnBf16Cfg {
+  static constexpr int kThreads = 256;
+  static constexpr int kCtasPerSm = 2;
+  static constexpr int kSmemBytes = 1024 + 3 * kTileBytes;
+  // Registers: two CTAs share the file, 128 per thread at launch; setmaxnreg moves them from the service warps
+  // to the softmax warps.  The move waits without bound for registers the CTA does not own, so the sum is
+  // checked here and the compiled register count is checked on the host before the first launch.
+  static constexpr int kRegsBase = 128;
+  static constexpr int kRegsService = 56;
+  static constexpr int kRegsSoftmax = 200;
+  static constexpr int kRegsAfterMove = 128 * kRegsService + 128 * kRegsSoftmax;
+  static_assert(kRegsAfterMove <= kThreads * kRegsBase, "register budget: setmaxnreg.inc would wait forever");
+  static_assert(kThreads * kRegsBase * kCtasPerSm <= 65536, "two CTAs must fit the register file");
+};
+
+// Masked iterations (diagonal blocks, correction chunks -- the minority): overwrite the hidden logits of this
+// thread's row with -inf in TMEM, so that the softmax step itself carries no mask logic.  Column j stays
+// visible iff j <= tok_lim and bit j of the 128-bit mask (32 bits per word) is set.  Not inlined: it is off the
+// common path and four times 32 unrolled selects are a lot of code.
+__device__ __noinline__ void mask_row(uint32_t s_addr, int tok_lim, uint32_t cm0, uint32_t cm1, uint32_t cm2,
+                                      uint32_t cm3) {
+#pragma unroll 1
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t cmk = k == 0 ? cm0 : k == 1 ? cm1 : k == 2 ? cm2 : cm3;
+    const bool all_vis = (k * 32 + 31 <= tok_lim) && (cmk == 0xffffffffu);
+    if (__all_sync(0xffffffffu, all_vis)) continue;   // TMEM accesses are warp-wide: decide per warp
+    uint32_t rr[32];
+    tmem_ld32(s_addr + k * 32, rr);
+    tmem_wait_ld();
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+      const bool vis = (k * 32 + j <= tok_lim) && ((cmk >> j) & 1u);
+      rr[j] = vis ? rr[j] : 0xff800000u;  // -inf
+    }
+    tmem_st32(s_addr + k * 32, rr);
+  }
+  tmem_wait_st();
+}
+
+// The thread's whole logit row (raw, unscaled) into registers, and its maximum: all four TMEM loads in flight,
+// chains of three-input maxima.
+__device__ __forceinline__ float row_load_max(uint32_t s_addr, uint32_t (&x)[128]) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k) tmem_ld32(s_addr + k * 32, reinterpret_cast<uint32_t(&)[32]>(x[k * 32]));
+  tmem_wait_ld();
+  float mx8[16];
+#pragma unroll
+  for (int c = 0; c < 16; ++c) {
+    const float* v = reinterpret_cast<const float*>(&x[c * 8]);
+    mx8[c] = fmaxf(max3(max3(v[0], v[1], v[2]), v[3], v[4]), max3(v[5], v[6], v[7]));
+  }
+#pragma unroll
+  for (int c = 0; c < 5; ++c) mx8[c] = max3(mx8[3 * c], mx8[3 * c + 1], mx8[3 * c + 2]);
+  return fmaxf(max3(mx8[0], mx8[1], mx8[2]), max3(mx8[3], mx8[4], mx8[15]));
+}
+
+// p = 2^(x * cs + neg_m) for the 128 logits in registers, written as BF16 pairs to the 64 columns at p_addr.
+// Scaling and row sum use packed fp32x2 instructions.  After the first 64 probabilities the thread arrives on
+// half_ready.  Returns the row sum.
+__device__ __forceinline__ float row_exp(const uint32_t (&x)[128], uint32_t p_addr, float cs, float neg_m,
+                                         uint64_t* half_ready) {
+  const uint64_t cs2 = f2_pack(cs, cs), nm2 = f2_pack(neg_m, neg_m);
+  uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};   // four independent (lo, hi) accumulators, +0.0f bit patterns
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      const uint64_t x2 =
+          f2_fma(f2_pack(__uint_as_float(x[k * 32 + 2 * j]), __uint_as_float(x[k * 32 + 2 * j + 1])), cs2, nm2);
+      float x0, x1;
+      f2_unpack(x2, x0, x1);
+      const float p0 = ex2(x0), p1 = ex2(x1);
+      sum2[j & 3] = f2_add(sum2[j & 3], f2_pack(p0, p1));
+      pk[j] = pack_bf16x2(p0, p1);
+    }
+    tmem_st16(p_addr + k * 16, pk);
+    if (k < 3) {   // a quarter of P: O += P V may run its next two k-steps
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&half_ready[k]);
+    }
+  }
+  float a0, a1;
+  f2_unpack(f2_add(f2_add(sum2[0], sum2[1]), f2_add(sum2[2], sum2[3])), a0, a1);
+  return a0 + a1;
+}
+
+__global__ void __launch_bounds__(AttnBf16Cfg::kThreads, AttnBf16Cfg::kCtasPerSm)
+sparse_attn_bf16_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
+                        const __grid_constant__ CUtensorMap map_kbar, const __grid_constant__ CUtensorMap map_vbar,
+                        AttnArgs A, DevParams P) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sQ = smem;
+  uint8_t* sK = smem + kTileBytes;
+  uint8_t* sV = sK + kTileBytes;
+
+  __shared__ TileInfo info[2];
+  __shared__ uint32_t sel_bits[kMaxBlocks / 32];
+  __shared__ uint64_t info_full[2], info_empty[2], q_full, q_empty;
+  // Every barrier below completes exactly once per iteration; with G the iteration's index counted over the
+  // whole kernel, the phase that belongs to iteration G has parity G & 1.
+  __shared__ uint64_t k_full, v_full;
+  __shared__ uint64_t s_done;    // S = Q K^T (G) has completed: the logits are in TMEM, the K stage is free --
+                                 // and, MMAs completing in issue order, O += P V (G-1) is in O
+  __shared__ uint64_t pv_done;   // O += P V (G) has completed: the V stage is free, O holds iteration G
+  __shared__ uint64_t p_ready[4];   // quarter q (32 probabilities of every row) of P (G) is in TMEM
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  WaitCtx ctx{A.status, &abort_flag};
+
+  if (tid == 0) {
+    abort_flag = 0;
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&info_full[i], 1);
+      mbar_init(&info_empty[i], 2 + 128);   // producer, issuer, softmax threads
+    }
+    mbar_init(&q_full, 64);
+    mbar_init(&q_empty, 1);
+    mbar_init(&k_full, 1);
+    mbar_init(&v_full, 1);
+    mbar_init(&s_done, 1);
+    mbar_init(&pv_done, 1);
+    for (int i = 0; i < 4; ++i) mbar_init(&p_ready[i], 128);
+    fence_barrier_init();
+  }
+  // K / V stages start zeroed: rows of pages past the end of a sequence are never loaded, and whatever sits
+  // there is multiplied by probabilities that are exactly zero, so it must be finite.
+  for (int i = tid; i < 2 * kTileBytes / 16; i += AttnBf16Cfg::kThreads)
+    reinterpret_cast<uint4*>(sK)[i] = make_uint4(0, 0, 0, 0);
+  if (warp == 5) {
+    tmem_alloc(&tmem_base_s, 256);
+    tmem_relinquish();
+  }
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base_s;
+  const int g = P.group;
+
+  if (warp >= 6) {
+    // =============================== unit set-up + Q staging ===============================
+    setmaxnreg_dec<AttnBf16Cfg::kRegsService>();
+    const int t64 = tid - 32 * 6;
+    for (int it = 0;; ++it) {
+      const int slot = it & 1;
+      if (it >= 2) mbar_wait(&info_empty[slot], ((it >> 1) - 1) & 1, ctx, 201);
+      TileInfo& ti = info[slot];
+      if (t64 == 0) {
+        const int w = atomicAdd(A.work_counter, 1);
+        if (w < P.nseg) {
+          const int seg = A.order[w];
+          ti.sg = A.segs[seg];
+          ti.valid = 1;
+          ti.dense = (A.seg_count == nullptr);
+          int T = ti.dense ? ti.sg.J_hi + 1 : A.seg_count[seg];
+          if (T < 0 || T > ti.sg.J_hi + 1) {  // malformed count: clamp so every loop stays bounded
+            atomicOr(A.status + ST_BAD_LIST, 1);
+            T = max(0, min(T, ti.sg.J_hi + 1));
+          }
+          ti.T = T;
+          ti.nchunk = 0;
+        } else {
+          ti.valid = 0;
+        }
+      }
+      named_bar_sync(2, 64);
+      const bool valid = ti.valid != 0;
+      if (valid && !ti.dense) {
+        const SegInfo& sg = ti.sg;
+        const int32_t* list = A.blk_idx + sg.off;
+        const int T = ti.T;
+        const int nwords = (sg.J_lo + 31) >> 5;
+        const bool corr = P.use_correction != 0;
+        if (corr)
+          for (int w = t64; w < nwords; w += 64) sel_bits[w] = 0u;
+        named_bar_sync(2, 64);
+        bool bad = false;
+        for (int k = t64; k < T; k += 64) {
+          const int J = list[k];
+          if (J < 0 || J > sg.J_hi || (k > 0 && list[k - 1] >= J)) bad = true;
+          if (corr && J >= 0 && J < sg.J_lo) atomicOr(&sel_bits[J >> 5], 1u << (J & 31));
+        }
+        if (bad) atomicOr(A.status + ST_BAD_LIST, 1);
+        named_bar_sync(2, 64);
+        if (corr) {
+          const int nch = (sg.J_lo + 127) >> 7;
+          for (int c = t64; c < nch; c += 64) {
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+              const int first = c * 128 + w * 32;
+              uint32_t validm = 0u;
+              if (first + 32 <= sg.J_lo) validm = 0xffffffffu;
+              else if (first < sg.J_lo) validm = (1u << (sg.J_lo - first)) - 1u;
+              ti.todo[c][w] = (first < sg.J_lo ? ~sel_bits[first >> 5] : 0u) & validm;
+            }
+          }
+          named_bar_sync(2, 64);
+          if (t64 == 0) {
+            int n = 0;
+            for (int c = 0; c < nch; ++c)
+              if (ti.todo[c][0] | ti.todo[c][1] | ti.todo[c][2] | ti.todo[c][3]) ti.chunk_id[n++] = c;
+            ti.nchunk = n;
+          }
+        }
+      }
+      named_bar_sync(2, 64);
+      if (t64 == 0) mbar_arrive(&info_full[slot]);
+      if (!valid) break;
+      // Q tile: wait until every S = Q K^T of the previous unit has completed, then overwrite
+      if (it >= 1) mbar_wait(&q_empty, (it - 1) & 1, ctx, 202);
+      load_q_tile_async(sQ, A.q, ti.sg, P, t64, 64);
+      fence_proxy_async();
+      mbar_arrive(&q_full);
+    }
+  } else if (warp == 4) {
+    // =============================== TMA producer ===============================
+    setmaxnreg_dec<AttnBf16Cfg::kRegsService>();
+    if (lane == 0) {
+      tma_prefetch_desc(&map_k);
+      tma_prefetch_desc(&map_v);
+      tma_prefetch_desc(&map_kbar);
+      tma_prefetch_desc(&map_vbar);
+    }
+    uint32_t G = 0;
+    const uint64_t keep = l2_policy_evict_last();   // K / V pages and pooled means: shared by many tiles
+    const int ppb = P.pages_per_block, psz = P.page_size;
+    for (int it = 0;; ++it) {
+      const int slot = it & 1;
+      mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 301);
+      const TileInfo& ti = info[slot];
+      if (!ti.valid) break;
+      const SegInfo& sg = ti.sg;
+      const int T = ti.T, n_it = T + ti.nchunk;
+      const int32_t* list = A.blk_idx + sg.off;
+      const int32_t* pt = A.page_table + (size_t)sg.b * P.max_pages_per_seq;
+      // page id of this lane's page of exact iteration i (-1: past the end of the sequence, or not an exact
+      // iteration).  Fetched one iteration ahead: list entry -> page-table entry are two dependent global loads.
+      auto fetch_pid = [&](int i) -> int {
+        if (i >= T || lane >= ppb) return -1;
+        int J = ti.dense ? sg.J_hi - i : list[T - 1 - i];
+        J = max(0, min(J, sg.J_hi));
+        if (J * kBlock + lane * psz >= sg.Lk) return -1;
+        int pid = pt[J * ppb + lane];
+        if (pid < 0 || pid >= P.num_pages) {
+          atomicOr(A.status + ST_BAD_LIST, 2);
+          pid = -1;
+        }
+        return pid;
+      };
+      int pid_next = fetch_pid(0);
+      for (int i = 0; i < n_it; ++i, ++G) {
+        const int pid = pid_next;
+        pid_next = fetch_pid(i + 1);
+        if (i < T) {
+          const int nvalid = __popc(__ballot_sync(0xffffffffu, pid >= 0));
+          const uint32_t bytes = (uint32_t)nvalid * psz * 256u;
+          if (G >= 1) mbar_wait(&s_done, (G - 1) & 1, ctx, 302);   // K stage free
+          if (lane == 0) mbar_arrive_expect_tx(&k_full, bytes);
+          __syncwarp();
+          if (pid >= 0) {
+            tma_load_3d_hint(sK + lane * psz * 128, &map_k, &k_full, 0, sg.h, pid * psz, keep);
+            tma_load_3d_hint(sK + 16384 + lane * psz * 128, &map_k, &k_full, 64, sg.h, pid * psz, keep);
+          }
+          if (G >= 1) mbar_wait(&pv_done, (G - 1) & 1, ctx, 303);  // V stage free
+          if (lane == 0) mbar_arrive_expect_tx(&v_full, bytes);
+          __syncwarp();
+          if (pid >= 0) {
+            tma_load_3d_hint(sV + lane * psz * 128, &map_v, &v_full, 0, sg.h, pid * psz, keep);
+            tma_load_3d_hint(sV + 16384 + lane * psz * 128, &map_v, &v_full, 64, sg.h, pid * psz, keep);
+          }
+        } else {
+          const int row0 = sg.blk_off + ti.chunk_id[i - T] * 128;
+          if (G >= 1) mbar_wait(&s_done, (G - 1) & 1, ctx, 304);
+          if (lane == 0) {
+            mbar_arrive_expect_tx(&k_full, kTileBytes);
+            tma_load_3d_hint(sK, &map_kbar, &k_full, 0, sg.h, row0, keep);
+            tma_load_3d_hint(sK + 16384, &map_kbar, &k_full, 64, sg.h, row0, keep);
+          }
+          if (G >= 1) mbar_wait(&pv_done, (G - 1) & 1, ctx, 305);
+          if (lane == 0) {
+            mbar_arrive_expect_tx(&v_full, kTileBytes);
+            tma_load_3d_hint(sV, &map_vbar, &v_full, 0, sg.h, row0, keep);
+            tma_load_3d_hint(sV + 16384, &map_vbar, &v_full, 64, sg.h, row0, keep);
+          }
+          __syncwarp();
+        }
+      }
+      if (lane == 0) mbar_arrive(&info_empty[slot]);
+    }
+  } else if (warp == 5) {
+    // =============================== UMMA issuer ===============================
+    setmaxnreg_dec<AttnBf16Cfg::kRegsService>();
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = make_idesc(128, 128, 1, 1, 0, 0);
+      constexpr uint32_t idesc_pv = make_idesc(128, 128, 1, 1, 0, 1);
+      const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+      uint32_t G = 0;
+      for (int it = 0;; ++it) {
+        const int slot = it & 1;
+        mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 403);
+        const TileInfo& ti = info[slot];
+        if (!ti.valid) break;
+        const int n_it = ti.T + ti.nchunk;
+        mbar_wait(&q_full, it & 1, ctx, 404);
+        for (int i = 0; i < n_it; ++i, ++G) {
+          // S = Q K^T (G).  The S columns are free: O += P V (G-1), which read P out of them, was issued before.
+          mbar_wait(&k_full, G & 1, ctx, 405);
+          tc_fence_after();
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+            const uint64_t ad = make_smem_desc_sw128(q_addr + off, 16, 1024);
+            const uint64_t bd = make_smem_desc_sw128(k_addr + off, 16, 1024);
+            umma_f16_ss(tmem, ad, bd, idesc_qk, ks > 0);
+          }
+          umma_commit(&s_done);
+          if (i == n_it - 1) umma_commit(&q_empty);
+          // O += P V (G)
+          mbar_wait(&v_full, G & 1, ctx, 402);
+#pragma unroll
+          for (int h = 0; h < 4; ++h) {   // as each quarter of P arrives
+            mbar_wait(&p_ready[h], G & 1, ctx, 401);
+            tc_fence_after();
+#pragma unroll
+            for (int ks = 2 * h; ks < 2 * h + 2; ++ks) {
+              const uint64_t bd = make_smem_desc_sw128(v_addr + ks * 2048, 16384, 1024);
+              umma_f16_ts(tmem + 128, tmem + ks * 8, bd, idesc_pv, (i > 0) || ks > 0);
+            }
+          }
+          umma_commit(&pv_done);
+        }
+        if (n_it == 0) umma_commit(&q_empty);  // empty list: nothing read Q, release it at once
+        mbar_arrive(&info_empty[slot]);
+      }
+    }
+  } else {
+    // =============================== softmax warpgroup + epilogue ===============================
+    setmaxnreg_inc<AttnBf16Cfg::kRegsSoftmax>();
+    const int row = warp * 32 + lane;
+    const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t s_addr = lane_base;         // S; P overwrites its first 64 columns
+    const uint32_t o_addr = lane_base + 128;
+    uint32_t G = 0;
+#ifdef FP2_TIMING
+    uint32_t ta[5] = {0, 0, 0, 0, 0}, tl = (uint32_t)clock(), tn = 0;
+#define FP2_T(k) { uint32_t n_ = (uint32_t)clock(); ta[k] += (n_ - tl) >> 3; tl = n_; }
+#else
+#define FP2_T(k)
+#endif
+    const uint64_t stream_pol = l2_policy_evict_first();   // outputs are written once and not read here
+    for (int it = 0;; ++it) {
+      const int slot = it & 1;
+      mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 501);
+      const TileInfo& ti = info[slot];
+      if (!ti.valid) break;
+      const int T = ti.T, n_it = T + ti.nchunk;
+      const bool dense = ti.dense != 0;
+      const int J_hi = ti.sg.J_hi, J_lo = ti.sg.J_lo;
+      const int32_t* list = A.blk_idx + ti.sg.off;
+      const int r = ti.sg.r0 + row;
+      const int pos = ti.sg.pre + r / g;
+      const float cs_all = P.scale_log2;
+      float m = -INFINITY, l = 0.f;
+      // block id of the next exact iteration, fetched one iteration ahead
+      int J_next = (!dense && T > 0) ? list[T - 1] : 0;
+      for (int i = 0; i < n_it; ++i, ++G) {
+        // iteration kind and masks
+        bool need_mask = false;
+        int tok_lim = 1 << 30;     // exact block: columns j with j <= tok_lim are visible
+        uint32_t cm0 = 0xffffffffu, cm1 = 0xffffffffu, cm2 = 0xffffffffu, cm3 = 0xffffffffu;
+        float shift = 0.f;
+        if (i < T) {
+          int J = dense ? J_hi - i : J_next;
+          if (!dense && i + 1 < T) J_next = list[T - 2 - i];
+          J = max(0, min(J, J_hi));
+          need_mask = J >= J_lo;
+          tok_lim = pos - J * kBlock;
+        } else {
+          const int c = ti.chunk_id[i - T];
+          cm0 = ti.todo[c][0];
+          cm1 = ti.todo[c][1];
+          cm2 = ti.todo[c][2];
+          cm3 = ti.todo[c][3];
+          shift = 7.0f;  // log2(128): one pooled row stands for a full block (Eq. 6)
+          need_mask = true;
+        }
+        FP2_T(0);
+        mbar_wait(&s_done, G & 1, ctx, 502);
+        tc_fence_after();
+        FP2_T(1);
+        if (need_mask) mask_row(s_addr, tok_lim, cm0, cm1, cm2, cm3);
+        uint32_t x[128];
+        const float mx = fmaf(row_load_max(s_addr, x), cs_all, shift);  // cs > 0: scaling commutes with the maximum
+        FP2_T(2);
+        const float m_new = fmaxf(m, mx);
+        // lazy rescale: only when some row of the warp moved its maximum by more than 2^8.  O is at rest: the
+        // MMAs complete in issue order, so S (G) in TMEM means O += P V (G-1) has been added.
+        if (__any_sync(0xffffffffu, m_new > m + 8.0f)) {
+          const float f = (m == -INFINITY) ? 0.f : ex2(m - m_new);
+          if (i > 0) {
+#pragma unroll 1
+            for (int k = 0; k < 4; ++k) {
+              uint32_t rr[32];
+              tmem_ld32(o_addr + k * 32, rr);
+              tmem_wait_ld();
+#pragma unroll
+              for (int j = 0; j < 32; ++j) rr[j] = __float_as_uint(__uint_as_float(rr[j]) * f);
+              tmem_st32(o_addr + k * 32, rr);
+            }
+          }
+          l *= f;
+          m = m_new;
+        }
+        // a row with nothing visible so far has m = -inf and only -inf logits: exponent against 0 -> zeros
+        const float neg_m = (m == -INFINITY) ? shift : shift - m;
+        FP2_T(3);
+        l += row_exp(x, s_addr, cs_all, neg_m, &p_ready[0]);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&p_ready[3]);
+        FP2_T(4);
+#ifdef FP2_TIMING
+        ++tn;
+#endif
+      }
+      // ------------------------------ epilogue ------------------------------
+      const SegInfo& sg = ti.sg;
+      const float inv = l > 0.f ? 1.0f / l : 0.f;
+      const bool have_o = n_it >= 1;
+      const bool row_ok = row < sg.nrows;
+      const size_t tok = (size_t)sg.q_tok0 + r / g;
+      const int head = sg.h * g + r % g;
+      __nv_bfloat16* orow = A.out + (tok * P.num_q_heads + head) * kHeadDim;
+      if (have_o) {
+        mbar_wait(&pv_done, (G - 1) & 1, ctx, 503);   // O += P V of the unit's last iteration
+        tc_fence_after();
+      }
+#pragma unroll 1
+      for (int k = 0; k < 4; ++k) {
+        uint32_t a0[32];
+        if (have_o) {
+          tmem_ld32(o_addr + k * 32, a0);
+          tmem_wait_ld();
+        }
+        uint32_t o[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float v0 = have_o ? __uint_as_float(a0[2 * j]) * inv : 0.f;
+          const float v1 = have_o ? __uint_as_float(a0[2 * j + 1]) * inv : 0.f;
+          o[j] = pack_bf16x2(v0, v1);
+        }
+        if (row_ok) {   // 32-byte stores: every instruction writes whole sectors
+          st_global_v8(orow + k * 32, &o[0], stream_pol);
+          st_global_v8(orow + k * 32 + 16, &o[8], stream_pol);
+        }
+      }
+      if (row_ok && A.lse != nullptr)
+        A.lse[(size_t)head * P.total_q + tok] = (m + log2f(l)) * 0.6931471805599453f;
+      tc_fence_before();
+      mbar_arrive(&info_empty[slot]);
+    }
+#ifdef FP2_TIMING
+    if (blockIdx.x < 2 && tid == 0)
+      printf("cta %d iters %u: loop-top %u wait_s %u mask+load+max %u rescale %u exp+store+arrive %u\n", blockIdx.x, tn,
+             ta[0] * 8 / tn, ta[1] * 8 / tn, ta[2] * 8 / tn, ta[3] * 8 / tn, ta[4] * 8 / tn);
+#endif
+  }
+  // teardown: on the normal path every barrier has been consumed; after an abort give in-flight copies time
+  if (abort_flag) __nanosleep(2000000);
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem, 256);
+}
+
+}  // namespace fp2
