@@ -28,6 +28,8 @@
 
 namespace fp2 {
 
+constexpr int kPParts = 4;   // P is handed to the issuer in this many column slices (4 or 8)
+
 struct AttnBf16Cfg {
   static constexpr int kThreads = 256;
   static constexpr int kCtasPerSm = 2;
@@ -88,27 +90,28 @@ __device__ __forceinline__ float row_load_max(uint32_t s_addr, uint32_t (&x)[128
 // Scaling and row sum use packed fp32x2 instructions.  After the first 64 probabilities the thread arrives on
 // half_ready.  Returns the row sum.
 __device__ __forceinline__ float row_exp(const uint32_t (&x)[128], uint32_t p_addr, float cs, float neg_m,
-                                         uint64_t* half_ready) {
+                                         uint64_t* part_ready) {
   const uint64_t cs2 = f2_pack(cs, cs), nm2 = f2_pack(neg_m, neg_m);
   uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};   // four independent (lo, hi) accumulators, +0.0f bit patterns
 #pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    uint32_t pk[16];
+  for (int k = 0; k < kPParts; ++k) {
+    constexpr int W = 64 / kPParts;   // packed registers (= P columns) per part
+    uint32_t pk[W];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const uint64_t x2 =
-          f2_fma(f2_pack(__uint_as_float(x[k * 32 + 2 * j]), __uint_as_float(x[k * 32 + 2 * j + 1])), cs2, nm2);
+    for (int j = 0; j < W; ++j) {
+      const int c = k * 2 * W + 2 * j;
+      const uint64_t x2 = f2_fma(f2_pack(__uint_as_float(x[c]), __uint_as_float(x[c + 1])), cs2, nm2);
       float x0, x1;
       f2_unpack(x2, x0, x1);
       const float p0 = ex2(x0), p1 = ex2(x1);
       sum2[j & 3] = f2_add(sum2[j & 3], f2_pack(p0, p1));
       pk[j] = pack_bf16x2(p0, p1);
     }
-    tmem_st16(p_addr + k * 16, pk);
-    if (k < 3) {   // a quarter of P: O += P V may run its next two k-steps
+    tmem_st_cols(p_addr + k * W, pk);
+    if (k + 1 < kPParts) {   // a part of P: O += P V may run its next k-steps
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&half_ready[k]);
+      mbar_arrive(&part_ready[k]);
     }
   }
   float a0, a1;
@@ -135,7 +138,7 @@ sparse_attn_bf16_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
   __shared__ uint64_t s_done;    // S = Q K^T (G) has completed: the logits are in TMEM, the K stage is free --
                                  // and, MMAs completing in issue order, O += P V (G-1) is in O
   __shared__ uint64_t pv_done;   // O += P V (G) has completed: the V stage is free, O holds iteration G
-  __shared__ uint64_t p_ready[4];   // quarter q (32 probabilities of every row) of P (G) is in TMEM
+  __shared__ uint64_t p_ready[kPParts];   // slice q (128 / kPParts probabilities of every row) of P (G) is in TMEM
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
 
@@ -154,7 +157,7 @@ sparse_attn_bf16_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
     mbar_init(&v_full, 1);
     mbar_init(&s_done, 1);
     mbar_init(&pv_done, 1);
-    for (int i = 0; i < 4; ++i) mbar_init(&p_ready[i], 128);
+    for (int i = 0; i < kPParts; ++i) mbar_init(&p_ready[i], 128);
     fence_barrier_init();
   }
   // K / V stages start zeroed: rows of pages past the end of a sequence are never loaded, and whatever sits
@@ -353,11 +356,11 @@ sparse_attn_bf16_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
           // O += P V (G)
           mbar_wait(&v_full, G & 1, ctx, 402);
 #pragma unroll
-          for (int h = 0; h < 4; ++h) {   // as each quarter of P arrives
+          for (int h = 0; h < kPParts; ++h) {   // as each slice of P arrives
             mbar_wait(&p_ready[h], G & 1, ctx, 401);
             tc_fence_after();
 #pragma unroll
-            for (int ks = 2 * h; ks < 2 * h + 2; ++ks) {
+            for (int ks = (8 / kPParts) * h; ks < (8 / kPParts) * (h + 1); ++ks) {
               const uint64_t bd = make_smem_desc_sw128(v_addr + ks * 2048, 16384, 1024);
               umma_f16_ts(tmem + 128, tmem + ks * 8, bd, idesc_pv, (i > 0) || ks > 0);
             }
@@ -452,7 +455,7 @@ sparse_attn_bf16_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_
         l += row_exp(x, s_addr, cs_all, neg_m, &p_ready[0]);
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&p_ready[3]);
+        mbar_arrive(&p_ready[kPParts - 1]);
         FP2_T(4);
 #ifdef FP2_TIMING
         ++tn;
