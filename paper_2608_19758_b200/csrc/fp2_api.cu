@@ -14,7 +14,6 @@
 #include "pool_kv.cuh"
 #include "score_select.cuh"
 #include "sparse_attn.cuh"
-#include "sparse_attn_bf16.cuh"
 
 using namespace fp2;
 
@@ -35,7 +34,7 @@ struct fp2_plan {
   SegInfo* d_segs;
   int32_t* d_blk_off;
   // workspace layout (byte offsets)
-  int64_t ws_status, ws_counter, ws_khi, ws_klo, ws_vbar, ws_order, ws_hist, ws_bytes;
+  int64_t ws_status, ws_counter, ws_khi, ws_klo, ws_vbar, ws_k8hi, ws_k8lo, ws_order, ws_hist, ws_bytes;
   EncodeTiledFn encode;
   int32_t last_launches;
   bool attrs_set;
@@ -174,6 +173,11 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
   pl->ws_khi = o;  o += pooled;
   pl->ws_klo = o;  o += pooled;
   pl->ws_vbar = o; o += pooled;
+  // FP8 plans: the pooled keys once more, as an e4m3 hi + lo pair in raw units (correction chunks of the
+  // attention kernel)
+  const int64_t pooled8 = p->dtype == FP2_FP8_E4M3 ? align_up(nblk_tot * p->num_kv_heads * kHeadDim, 1024) : 0;
+  pl->ws_k8hi = o; o += pooled8;
+  pl->ws_k8lo = o; o += pooled8;
   pl->ws_order = o; o += align_up(4 * (pl->nseg > 0 ? pl->nseg : 1), 1024);
   pl->ws_hist = o;  o += align_up(4 * ((int64_t)p->num_kv_heads * kCountBuckets + 1), 1024);
   pl->ws_bytes = o;
@@ -242,16 +246,16 @@ static fp2_status set_attrs(fp2_plan* pl) {
                            kScoreSmemBytes) != cudaSuccess ||
       cudaFuncSetAttribute(score_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kScoreSmemBytes) != cudaSuccess ||
-      cudaFuncSetAttribute(sparse_attn_bf16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           AttnBf16Cfg::kSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(sparse_attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           AttnCfg<false>::kSmemBytes) != cudaSuccess ||
       cudaFuncSetAttribute(sparse_attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            AttnCfg<true>::kSmemBytes) != cudaSuccess)
     return FP2_ERR_CUDA;
   // The attention kernels move registers between warps with setmaxnreg, whose wait is unbounded: launch only
   // if the compiled kernels really own the registers the move assumes.
   cudaFuncAttributes fa;
-  if (cudaFuncGetAttributes(&fa, sparse_attn_bf16_kernel) != cudaSuccess) return FP2_ERR_CUDA;
-  if (fa.numRegs * AttnBf16Cfg::kThreads < AttnBf16Cfg::kRegsAfterMove) return FP2_ERR_UNSUPPORTED;
+  if (cudaFuncGetAttributes(&fa, sparse_attn_kernel<false>) != cudaSuccess) return FP2_ERR_CUDA;
+  if (fa.numRegs * AttnCfg<false>::kThreads < AttnCfg<false>::kRegsAfterMove) return FP2_ERR_UNSUPPORTED;
   if (cudaFuncGetAttributes(&fa, sparse_attn_kernel<true>) != cudaSuccess) return FP2_ERR_CUDA;
   if (fa.numRegs * AttnCfg<true>::kThreads < AttnCfg<true>::kRegsAfterMove) return FP2_ERR_UNSUPPORTED;
   pl->attrs_set = true;
@@ -282,10 +286,10 @@ static fp2_status launch_pool(fp2_plan* pl, const void* k, const void* v, const 
   __nv_bfloat16* vb = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_vbar);
   if (pl->dev.fp8)
     pool_kv_kernel<true><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, lk, pl->d_blk_off, ks, vs,
-                                               pl->dev, khi, klo, vb);
+                                               pl->dev, khi, klo, vb, ws + pl->ws_k8hi, ws + pl->ws_k8lo);
   else
     pool_kv_kernel<false><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, lk, pl->d_blk_off, ks, vs,
-                                                pl->dev, khi, klo, vb);
+                                                pl->dev, khi, klo, vb, nullptr, nullptr);
   pl->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
@@ -340,12 +344,18 @@ extern "C" fp2_status fp2_select_blocks(fp2_plan* pl, const void* q, const void*
 // ------------------------------------------------------------------------------------------------------
 // stage 2 (sparse and dense)
 // ------------------------------------------------------------------------------------------------------
-// BF16 attention: two 256-thread CTAs per SM, each a persistent worker on the shared work counter.
-static void launch_attn_bf16(fp2_plan* pl, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mkb,
-                             const CUtensorMap& mvb, const AttnArgs& a, cudaStream_t st) {
-  const int64_t workers = (int64_t)pl->num_sms * AttnBf16Cfg::kCtasPerSm;
+// Attention: two 256-thread CTAs per SM, each a persistent worker on the shared work counter.  mkb / mkb_lo:
+// pooled keys of the correction chunks (BF16: one BF16 array, mkb_lo unused; FP8: e4m3 hi and lo).
+static void launch_attn(fp2_plan* pl, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mkb,
+                        const CUtensorMap& mkb_lo, const CUtensorMap& mvb, const AttnArgs& a, cudaStream_t st) {
+  const int64_t workers = (int64_t)pl->num_sms * AttnCfg<false>::kCtasPerSm;
   const unsigned grid = (unsigned)(pl->nseg < workers ? pl->nseg : workers);
-  sparse_attn_bf16_kernel<<<grid, AttnBf16Cfg::kThreads, AttnBf16Cfg::kSmemBytes, st>>>(mk, mv, mkb, mvb, a, pl->dev);
+  if (pl->dev.fp8)
+    sparse_attn_kernel<true><<<grid, AttnCfg<true>::kThreads, AttnCfg<true>::kSmemBytes, st>>>(mk, mv, mkb, mkb_lo,
+                                                                                                 mvb, a, pl->dev);
+  else
+    sparse_attn_kernel<false><<<grid, AttnCfg<false>::kThreads, AttnCfg<false>::kSmemBytes, st>>>(
+        mk, mv, mkb, mkb_lo, mvb, a, pl->dev);
 }
 
 static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, const void* v, const int32_t* pt,
@@ -363,12 +373,19 @@ static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, cons
   if ((s = launch_order(pl, seg_count, ws, st)) != FP2_OK) return s;
   const bool fp8 = pl->dev.fp8 != 0;
   const int64_t slots = (int64_t)pl->prm.num_pages * pl->prm.page_size;
-  CUtensorMap mk, mv, mkb, mvb;
+  CUtensorMap mk, mv, mkb, mkb_lo, mvb;
   if (!make_map(pl, &mk, k, slots, pl->prm.num_kv_heads, pl->prm.page_size, fp8) ||
       !make_map(pl, &mv, v, slots, pl->prm.num_kv_heads, pl->prm.page_size, fp8) ||
-      !make_map(pl, &mkb, ws + pl->ws_khi, pl->nblk_tot, pl->prm.num_kv_heads, 128, false) ||
       !make_map(pl, &mvb, ws + pl->ws_vbar, pl->nblk_tot, pl->prm.num_kv_heads, 128, false))
     return FP2_ERR_CUDA;
+  if (fp8) {   // correction chunks: pooled keys as an e4m3 hi + lo pair
+    if (!make_map(pl, &mkb, ws + pl->ws_k8hi, pl->nblk_tot, pl->prm.num_kv_heads, 128, true) ||
+        !make_map(pl, &mkb_lo, ws + pl->ws_k8lo, pl->nblk_tot, pl->prm.num_kv_heads, 128, true))
+      return FP2_ERR_CUDA;
+  } else {
+    if (!make_map(pl, &mkb, ws + pl->ws_khi, pl->nblk_tot, pl->prm.num_kv_heads, 128, false)) return FP2_ERR_CUDA;
+    mkb_lo = mkb;
+  }
   AttnArgs a;
   a.q = reinterpret_cast<const uint8_t*>(q);
   a.page_table = pt;
@@ -381,12 +398,7 @@ static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, cons
   a.lse = lse;
   a.work_counter = reinterpret_cast<int*>(ws + pl->ws_counter);
   a.status = reinterpret_cast<int*>(ws + pl->ws_status);
-  const unsigned grid = (unsigned)(pl->nseg < pl->num_sms ? pl->nseg : pl->num_sms);
-  if (fp8)
-    sparse_attn_kernel<true><<<grid, AttnCfg<true>::kThreads, AttnCfg<true>::kSmemBytes, st>>>(mk, mv, mkb, mvb, a,
-                                                                                              pl->dev);
-  else
-    launch_attn_bf16(pl, mk, mv, mkb, mvb, a, st);
+  launch_attn(pl, mk, mv, mkb, mkb_lo, mvb, a, st);
   pl->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
@@ -484,7 +496,7 @@ extern "C" fp2_status fp2_dense_prefill_static(fp2_plan* pl, const void* q, cons
   a.work_counter = reinterpret_cast<int*>(sw + 64);
   a.status = reinterpret_cast<int*>(sw);
   // the dense path stages no pooled chunks: the two pooled-mean maps are never dereferenced
-  launch_attn_bf16(pl, mk, mv, mk, mv, a, st);
+  launch_attn(pl, mk, mv, mk, mk, mv, a, st);
   pl->last_launches = 4;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }

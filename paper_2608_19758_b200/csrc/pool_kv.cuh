@@ -6,9 +6,11 @@
 //   kbar_hi = bf16(mean k), kbar_lo = bf16(mean k - kbar_hi)   (hi + lo carries ~16 mantissa bits for the scorer)
 //   vbar    = bf16(mean v)
 // kbar_hi and vbar double as the operands of the correction chunks in the attention kernel.
-// FP8 inputs: the three arrays hold F16 instead of BF16 (both kernels downstream run their MMAs on F16 copies
-// of the raw e4m3 values): kbar_hi / kbar_lo = F16 pair of the de-scaled mean (mean of raw values x k_scale),
-// vbar = f16(mean of RAW v) -- v_scale is applied to the attention output.
+// FP8 inputs: the three arrays hold F16 instead of BF16: kbar_hi / kbar_lo = F16 pair of the de-scaled mean (mean
+// of raw values x k_scale) for the scorer, vbar = f16(mean of RAW v) -- v_scale is applied to the attention
+// output.  Two more arrays, e4m3 [nblk_tot, Hkv, 128] each, hold the mean of the RAW keys as a hi + lo pair
+// (hi = e4m3(mean), lo = e4m3(mean - hi): ~8 mantissa bits together) for the correction chunks of the attention
+// kernel, whose S = Q K^T runs on raw e4m3 operands.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -53,7 +55,9 @@ __global__ void __launch_bounds__(256, 4) pool_kv_kernel(const uint8_t* __restri
                                                          const float* __restrict__ v_scale, DevParams P,
                                                          __nv_bfloat16* __restrict__ kbar_hi,
                                                          __nv_bfloat16* __restrict__ kbar_lo,
-                                                         __nv_bfloat16* __restrict__ vbar) {
+                                                         __nv_bfloat16* __restrict__ vbar,
+                                                         uint8_t* __restrict__ kbar8_hi,
+                                                         uint8_t* __restrict__ kbar8_lo) {
   constexpr int ROW_BYTES = FP8 ? 128 : 256;
   constexpr int CHUNKS = ROW_BYTES / 16;       // 16-byte chunks per token row
   constexpr int EPC = FP8 ? 16 : 8;            // elements per chunk
@@ -104,8 +108,17 @@ __global__ void __launch_bounds__(256, 4) pool_kv_kernel(const uint8_t* __restri
 #pragma unroll
     for (int r = 0; r < ROWS_PER_PASS; ++r) s += red[r][c];
     float mean = s / (float)ntok;
-    if constexpr (FP8) mean *= (which == 0 ? k_scale[h] : 1.0f);
     const size_t o = ((size_t)gblk * P.num_kv_heads + h) * kHeadDim + c;
+    if constexpr (FP8) {
+      if (which == 0) {
+        // the attention kernel multiplies raw e4m3 queries with this pair in one FP8 MMA group each
+        const __nv_fp8_storage_t hi8 = __nv_cvt_float_to_fp8(mean, __NV_SATFINITE, __NV_E4M3);
+        const float hi8f = __half2float(__half(__nv_cvt_fp8_to_halfraw(hi8, __NV_E4M3)));
+        kbar8_hi[o] = hi8;
+        kbar8_lo[o] = __nv_cvt_float_to_fp8(mean - hi8f, __NV_SATFINITE, __NV_E4M3);
+        mean *= k_scale[h];
+      }
+    }
     if constexpr (FP8) {
       const __half hi16 = __float2half_rn(mean);
       if (which == 0) {

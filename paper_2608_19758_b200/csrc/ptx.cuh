@@ -63,7 +63,11 @@ __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, const 
   int spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if (((++spins) & 255) == 0) {
-      if (*ctx.abort) return;
+      if (*ctx.abort) {
+        // words 3..7: the wait each role (2xx .. 6xx) of an aborted CTA was found in (last writer wins)
+        if (where >= 200 && where < 700) ctx.status[3 + (where / 100 - 2)] = where;
+        return;
+      }
       if (clock64() - t0 > FP2_WAIT_CYCLES) {
         *ctx.abort = 1;
         if (atomicCAS(ctx.status + ST_TIMEOUT, 0, 1) == 0) ctx.status[ST_WHERE] = where;

@@ -83,19 +83,33 @@ __device__ __forceinline__ void load_q_tile_bf16(uint8_t* sQ, const uint8_t* __r
 // layout of the K / V rings.  nthr threads (a multiple of 8); eight consecutive threads take one row, so every quarter-warp reads
 // one whole 128-byte row (conflict-free).  Element order inside a row is preserved, so the same routine
 // serves K (K-major operand) and V (MN-major operand).
-__device__ __forceinline__ void widen_tile_f16(const uint8_t* raw, uint8_t* dst, int t, int nthr) {
-#pragma unroll 4
-  for (int i = t; i < kTileRows * 8; i += nthr) {
-    const int row = i >> 3, c = i & 7;        // c: 16-byte chunk = 16 elements d = 16c .. 16c+15
-    const uint4 v = *reinterpret_cast<const uint4*>(raw + sw128_offset(row, c));
-    const uint4 lo = make_uint4(e4m3x2_to_f16x2(v.x), e4m3x2_to_f16x2(v.x >> 16), e4m3x2_to_f16x2(v.y),
-                                e4m3x2_to_f16x2(v.y >> 16));
-    const uint4 hi = make_uint4(e4m3x2_to_f16x2(v.z), e4m3x2_to_f16x2(v.z >> 16), e4m3x2_to_f16x2(v.w),
-                                e4m3x2_to_f16x2(v.w >> 16));
-    uint8_t* half = dst + (c >> 2) * 16384;   // d < 64 -> first half
-    const int oc = (c & 3) * 2;               // chunk index inside the half (8 f16 per 16 bytes)
-    *reinterpret_cast<uint4*>(half + sw128_offset(row, oc)) = lo;
-    *reinterpret_cast<uint4*>(half + sw128_offset(row, oc + 1)) = hi;
+__device__ __forceinline__ void widen_chunk_f16(const uint4& v, uint8_t* dst, int row, int c) {
+  const uint4 lo = make_uint4(e4m3x2_to_f16x2(v.x), e4m3x2_to_f16x2(v.x >> 16), e4m3x2_to_f16x2(v.y),
+                              e4m3x2_to_f16x2(v.y >> 16));
+  const uint4 hi = make_uint4(e4m3x2_to_f16x2(v.z), e4m3x2_to_f16x2(v.z >> 16), e4m3x2_to_f16x2(v.w),
+                              e4m3x2_to_f16x2(v.w >> 16));
+  uint8_t* half = dst + (c >> 2) * 16384;   // d < 64 -> first half
+  const int oc = (c & 3) * 2;               // chunk index inside the half (8 f16 per 16 bytes)
+  *reinterpret_cast<uint4*>(half + sw128_offset(row, oc)) = lo;
+  *reinterpret_cast<uint4*>(half + sw128_offset(row, oc + 1)) = hi;
+}
+// Loads go in batches of eight ahead of the stores: raw and dst are both shared memory, and a load the compiler
+// cannot prove independent of the previous store waits for it (measured: 1260 cycles per tile with 128 threads
+// against 885 with the loads hoisted).
+__device__ __forceinline__ void widen_tile_f16(const uint8_t* __restrict__ raw, uint8_t* __restrict__ dst, int t,
+                                               int nthr) {
+  for (int i0 = t; i0 < kTileRows * 8; i0 += 8 * nthr) {
+    uint4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * nthr;
+      if (i < kTileRows * 8) v[u] = *reinterpret_cast<const uint4*>(raw + sw128_offset(i >> 3, i & 7));
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * nthr;   // row = i >> 3; c = i & 7: 16-byte chunk = 16 elements d = 16c .. 16c+15
+      if (i < kTileRows * 8) widen_chunk_f16(v[u], dst, i >> 3, i & 7);
+    }
   }
 }
 

@@ -2,74 +2,51 @@
 // persistent, warp-specialised, tcgen05 / TMEM / TMA.  The same kernel runs the dense path (implicit list
 // 0..J_hi, no correction).
 //
-// One CTA per SM loops over work units (sequence, KV head, packed query tile) taken from a work order
-// (KV-head-major, heaviest first) through a global counter.  For a unit with selected list idx[0..T) the
-// iteration sequence is the list traversed backwards (Eq. 17) followed by the non-empty correction chunks:
-// a correction chunk stages 128 consecutive pooled (kbar, vbar) rows exactly like a KV block, its logits are
-// shifted by log2(128) (every corrected block is full) and masked by todo = fully-visible & ~selected.
+// CTAs loop over work units (sequence, KV head, packed query tile) taken from a work order (KV-head-major,
+// heaviest first) through a global counter.  For a unit with selected list idx[0..T) the iteration sequence
+// is the list traversed backwards (Eq. 17) followed by the non-empty correction chunks: a correction chunk
+// stages 128 consecutive pooled (kbar, vbar) rows exactly like a KV block, its logits are shifted by log2(128)
+// (every corrected block is full) and masked by todo = fully-visible & ~selected.
 //
-// Roles:
-//   warps 0..4W-1   W = kWG softmax warpgroups (2 by default).  All work on EVERY iteration: warpgroup w owns
-//              logit columns [w 128/W, (w+1) 128/W) of all 128 rows (thread = row).  They exchange the row maximum
-//              through shared memory once per iteration; one accumulator O serves the whole tile (no merge at the
-//              end).  W = 4 (four warps per scheduler, 104 registers each) builds and passes parity but measured
-//              3 % (dense) to 10 % (sparse) slower at 32K than W = 2 with 224 registers.
-//   warp 4W    TMA producer: K / V pages through the page table into two rings (Eq. 22)
-//   warp 4W+1  UMMA issuer: S = Q K^T (SS), O += P V (P read from TMEM, V MN-major from shared memory)
-//   warps 4W+2, 4W+3  tile set-up: fetch the next unit, validate its list, build the correction masks, stage Q
-//   warps 4W+4..4W+7  (FP8 inputs only) widen raw e4m3 K / V tiles to F16 into the K / V rings
+// TWO small CTAs per SM.  Per 128x128 block the tensor pipe (two GEMMs) and the MUFU pipe (16384
+// exponentials) are each busy 1024 cycles, and a softmax step has several hundred cycles of latency around its
+// exponentials (TMEM load, row maximum, TMEM store, barrier hand-overs).  Two warpgroups that share one tile must
+// exchange row maxima and so move in lockstep: both are in their latency phase at the same time and the MUFU
+// pipe idles (that layout, one CTA of 12 warps per SM, measured 42-48 % tensor-pipe activity on the dense
+// path; this one 59 %).  Here every CTA has ONE softmax warpgroup that owns whole rows (thread = row, 128 logits
+// in registers), nothing crosses between the two CTAs of an SM, and they drift out of phase by themselves: while
+// one CTA's warps stream exponentials the other's wait for the tensor pipe, load logits or hand over P.
 //
-// TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512).  P (BF16 pairs) has its own
-// columns, so S = Q K^T of iteration i+2 may start as soon as the softmax of iteration i has read S -- it does
-// not wait for O += P V of iteration i.  Issue order: QK(0) QK(1) PV(0) QK(2) PV(1) ...  Per 128x128 block
-// the tensor pipe and the MUFU pipe are each busy 1024 cycles (ncu); how far the two overlap is what the
-// schedule decides.
+// One CTA: 256 threads, 96 KB of tile memory (Q, one K stage, one V stage), 256 TMEM columns:
+//   S [0,128)  logits of the iteration; P (16-bit pairs) overwrites its first 64 columns in place
+//   O [128,256)
+// Everything is single-buffered: S = Q K^T of iteration i+1 is issued behind O += P V of iteration i (which
+// reads P out of the S columns), the K tile of i+1 is requested when S = Q K^T (i) has completed and the V tile
+// when O += P V (i) has.  The other CTA of the SM fills the bubbles this leaves.  P is handed to the issuer in
+// kPParts column slices, so O += P V runs its first k-steps under the remaining exponentials.
+//
+// Roles: warps 0..3 softmax + epilogue; warp 4 TMA producer (Eq. 22); warp 5 UMMA issuer (and TMEM owner);
+// warps 6, 7 unit set-up (fetch the next unit, validate its list, build the correction masks, stage Q).
+//
+// FP8 inputs (Eq. 15; template parameter FP8): S = Q K^T runs as a kind::f8f6f4 MMA straight on the raw e4m3
+// tiles (Q and K both K-major, 128-byte rows, as cp.async / TMA write them), at twice the BF16 rate.  The
+// probabilities stay 16-bit -- a single e4m3 probability tile costs ~0.06 max-abs output error by itself -- so
+// O += P V is a kind::f16 MMA on F16 operands: P packed as F16, V widened (exactly) from its raw e4m3 tile into
+// the F16 V stage by the softmax warpgroup itself at the top of the iteration.  The per-head scales never touch
+// the operands: q_scale * k_scale multiplies the logits of a row, v_scale multiplies the output.  Correction
+// chunks: the pooled keys come as an e4m3 hi + lo pair in raw units (two accumulating MMA groups, ~8 mantissa
+// bits together), the pooled values as F16.  Tile memory: Q 16 KB, K 32 KB (one raw tile, or hi | lo of a
+// chunk), raw V 16 KB, F16 V 32 KB.
 #pragma once
 #include <cuda_bf16.h>
 #include "common.cuh"
 #include "ptx.cuh"
-#include "score_select.cuh"  // load_q_tile_bf16
+#include "score_select.cuh"  // load_q_tile_async
 
 namespace fp2 {
 
 constexpr int kTileBytes = 32768;   // one 128 x 128 tile of 16-bit elements
 constexpr int kRawBytes = 16384;    // one 128 x 128 tile of FP8 elements as TMA delivers it
-
-// FP8 inputs (Eq. 15) run through the same 16-bit pipeline: the producer lands raw e4m3 K / V tiles in a small
-// ring, a fourth warpgroup widens them to F16 (exact) into the K / V rings, and both GEMMs run as kind::f16
-// with F16 operands (Q widened when staged, P packed as F16).  The per-head scales never touch the operands:
-// q_scale * k_scale multiplies the logits of a row, v_scale multiplies the output.  A single e4m3 probability
-// tile, the other way to feed FP8 V to the tensor core, costs ~0.06 max-abs output error by itself.
-#ifndef FP2_SOFTMAX_WGS
-#define FP2_SOFTMAX_WGS 2
-#endif
-constexpr int kWG = FP2_SOFTMAX_WGS;      // softmax warpgroups; each owns 128 / kWG logit columns of every row
-constexpr int kCW = 128 / kWG;            // columns per warpgroup (64 or 32)
-constexpr int kSW = 4 * kWG;              // softmax warps; the service warps follow them
-static_assert(kWG == 2 || kWG == 4, "two or four softmax warpgroups");
-
-template <bool FP8>
-struct AttnCfg {
-  static constexpr int kThreads = 128 * kWG + 128 + (FP8 ? 128 : 0);
-  static constexpr int kNQ = FP8 ? 1 : 2;   // Q tiles in shared memory: two let the next unit's queries land while
-                                            // this unit is still being multiplied (FP8 has no room for a second)
-  static constexpr int kNK = 2;             // K ring stages (32 KB each).  Must stay 2: stage i % 2 is released by the
-                                            // same commit that publishes S buffer i % 2
-  static constexpr int kNV = 2;             // V ring stages
-  static constexpr int kNRaw = FP8 ? 3 : 0; // raw FP8 tile ring (16 KB each), K and V tiles alternate
-  static constexpr int kSmemBytes = 1024 + kTileBytes * (kNQ + kNK + kNV) + kNRaw * kRawBytes + 2048 * kWG;
-  // Registers.  The CTA is launched with kRegsBase registers per thread (what __launch_bounds__(kThreads, 1)
-  // lets ptxas use); setmaxnreg then moves registers from the service warps (kRegsService) to the softmax warps
-  // (kRegsSoftmax).  setmaxnreg.inc waits -- without bound -- until the CTA's own pool has the registers, so the
-  // total after the move must not exceed the launch allocation; the host checks the compiled register count
-  // against kRegsAfterMove before the first launch and refuses to launch otherwise.
-  static constexpr int kRegsBase = (65536 / kThreads) / 8 * 8;
-  static constexpr int kRegsService = (kWG == 4) ? 48 : 56;
-  static constexpr int kRegsSoftmax = (kWG == 4) ? (FP8 ? 96 : 104) : (FP8 ? 200 : 224);
-  static constexpr int kRegsAfterMove = (kThreads - 128 * kWG) * kRegsService + 128 * kWG * kRegsSoftmax;
-  static_assert(kRegsAfterMove <= kThreads * kRegsBase, "register budget: setmaxnreg.inc would wait forever");
-  static constexpr int kFmt = FP8 ? 0 : 1;  // UMMA kind::f16 operand format: 0 = F16, 1 = BF16
-};
 
 struct TileInfo {
   SegInfo sg;
@@ -97,21 +74,41 @@ struct AttnArgs {
   int* status;
 };
 
+constexpr int kPParts = 4;   // P is handed to the issuer in this many column slices (4 or 8)
+
+template <bool FP8>
+struct AttnCfg {
+  static constexpr int kThreads = 256;
+  static constexpr int kCtasPerSm = 2;
+  static constexpr int kSmemBytes = 1024 + 3 * kTileBytes;   // both dtypes: 96 KB of tiles
+  // Registers: two CTAs share the file, 128 per thread at launch; setmaxnreg moves them from the service warps
+  // to the softmax warps.  The move waits without bound for registers the CTA does not own, so the sum is
+  // checked here and the compiled register count is checked on the host before the first launch.
+  static constexpr int kRegsBase = 128;
+  static constexpr int kRegsService = 56;
+  static constexpr int kRegsSoftmax = 200;
+  static constexpr int kRegsAfterMove = (kThreads - 128) * kRegsService + 128 * kRegsSoftmax;
+  static_assert(kRegsAfterMove <= kThreads * kRegsBase, "register budget: setmaxnreg.inc would wait forever");
+  static_assert(kThreads * kRegsBase * kCtasPerSm <= 65536, "two CTAs must fit the register file");
+};
+
 // Masked iterations (diagonal blocks, correction chunks -- the minority): overwrite the hidden logits of this
-// thread's row with -inf in TMEM, so that the softmax step itself carries no mask logic (predicating the mask
-// into the softmax body cost 2.5x on every iteration, masked or not).  The thread owns kCW columns starting at
-// block column col0; column j stays visible iff j <= tok_lim and bit (j - col0) of cm (32 bits per word) is set.
-__device__ __forceinline__ void mask_cols(uint32_t s_addr, int col0, int tok_lim, const uint32_t* cm) {
-#pragma unroll
-  for (int k = 0; k < kCW / 32; ++k) {
-    const bool all_vis = (col0 + k * 32 + 31 <= tok_lim) && (cm[k] == 0xffffffffu);
+// thread's row with -inf in TMEM, so that the softmax step itself carries no mask logic.  Column j stays
+// visible iff j <= tok_lim and bit j of the 128-bit mask (32 bits per word) is set.  Not inlined: it is off the
+// common path and four times 32 unrolled selects are a lot of code.
+__device__ __noinline__ void mask_row(uint32_t s_addr, int tok_lim, uint32_t cm0, uint32_t cm1, uint32_t cm2,
+                                      uint32_t cm3) {
+#pragma unroll 1
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t cmk = k == 0 ? cm0 : k == 1 ? cm1 : k == 2 ? cm2 : cm3;
+    const bool all_vis = (k * 32 + 31 <= tok_lim) && (cmk == 0xffffffffu);
     if (__all_sync(0xffffffffu, all_vis)) continue;   // TMEM accesses are warp-wide: decide per warp
     uint32_t rr[32];
     tmem_ld32(s_addr + k * 32, rr);
     tmem_wait_ld();
 #pragma unroll
     for (int j = 0; j < 32; ++j) {
-      const bool vis = (col0 + k * 32 + j <= tok_lim) && ((cm[k] >> j) & 1u);
+      const bool vis = (k * 32 + j <= tok_lim) && ((cmk >> j) & 1u);
       rr[j] = vis ? rr[j] : 0xff800000u;  // -inf
     }
     tmem_st32(s_addr + k * 32, rr);
@@ -119,109 +116,86 @@ __device__ __forceinline__ void mask_cols(uint32_t s_addr, int col0, int tok_lim
   tmem_wait_st();
 }
 
-// This thread's kCW logit columns (raw, unscaled) into registers, and their maximum: all TMEM loads in flight,
+// The thread's whole logit row (raw, unscaled) into registers, and its maximum: all four TMEM loads in flight,
 // chains of three-input maxima.
-__device__ __forceinline__ float cols_row_max(uint32_t s_addr, uint32_t (&sv)[kCW]) {
+__device__ __forceinline__ float row_load_max(uint32_t s_addr, uint32_t (&x)[128]) {
 #pragma unroll
-  for (int k = 0; k < kCW / 32; ++k) tmem_ld32(s_addr + k * 32, reinterpret_cast<uint32_t(&)[32]>(sv[k * 32]));
+  for (int k = 0; k < 4; ++k) tmem_ld32(s_addr + k * 32, reinterpret_cast<uint32_t(&)[32]>(x[k * 32]));
   tmem_wait_ld();
-  float mx8[kCW / 8];
+  float mx8[16];
 #pragma unroll
-  for (int c = 0; c < kCW / 8; ++c) {
-    const float* v = reinterpret_cast<const float*>(&sv[c * 8]);
+  for (int c = 0; c < 16; ++c) {
+    const float* v = reinterpret_cast<const float*>(&x[c * 8]);
     mx8[c] = fmaxf(max3(max3(v[0], v[1], v[2]), v[3], v[4]), max3(v[5], v[6], v[7]));
   }
-  float r = fmaxf(fmaxf(mx8[0], mx8[1]), fmaxf(mx8[2], mx8[3]));
-  if constexpr (kCW == 64) r = fmaxf(r, fmaxf(fmaxf(mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
-  return r;
+#pragma unroll
+  for (int c = 0; c < 5; ++c) mx8[c] = max3(mx8[3 * c], mx8[3 * c + 1], mx8[3 * c + 2]);
+  return fmaxf(max3(mx8[0], mx8[1], mx8[2]), max3(mx8[3], mx8[4], mx8[15]));
 }
 
-// p = 2^(s * cs + neg_m) for this thread's kCW logits (still in the registers the maximum pass loaded them into),
-// written as 16-bit pairs to kCW / 2 columns at p_addr.  One TMEM read per logit: besides the latency, TMEM
-// loads of the softmax warps lengthen the time the tensor pipe takes to accept each MMA of the issuing thread.
-// Scaling and row sum use packed fp32x2 instructions.  Returns the row's partial sum.
+// p = 2^(x * cs + neg_m) for the 128 logits in registers, written as BF16 (F16) pairs to the 64 columns at p_addr.
+// Scaling and row sum use packed fp32x2 instructions.  After the first 64 probabilities the thread arrives on
+// half_ready.  Returns the row sum.
 template <bool F16>
-__device__ __forceinline__ float cols_row_exp(const uint32_t (&sv)[kCW], uint32_t p_addr, float cs, float neg_m) {
+__device__ __forceinline__ float row_exp(const uint32_t (&x)[128], uint32_t p_addr, float cs, float neg_m,
+                                         uint64_t* part_ready) {
   const uint64_t cs2 = f2_pack(cs, cs), nm2 = f2_pack(neg_m, neg_m);
   uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};   // four independent (lo, hi) accumulators, +0.0f bit patterns
 #pragma unroll
-  for (int k = 0; k < kCW / 32; ++k) {
-    uint32_t pk[16];
+  for (int k = 0; k < kPParts; ++k) {
+    constexpr int W = 64 / kPParts;   // packed registers (= P columns) per part
+    uint32_t pk[W];
 #pragma unroll
-    for (int j = 0; j < 16; ++j) {
-      const uint64_t x2 =
-          f2_fma(f2_pack(__uint_as_float(sv[k * 32 + 2 * j]), __uint_as_float(sv[k * 32 + 2 * j + 1])), cs2, nm2);
+    for (int j = 0; j < W; ++j) {
+      const int c = k * 2 * W + 2 * j;
+      const uint64_t x2 = f2_fma(f2_pack(__uint_as_float(x[c]), __uint_as_float(x[c + 1])), cs2, nm2);
       float x0, x1;
       f2_unpack(x2, x0, x1);
       const float p0 = ex2(x0), p1 = ex2(x1);
       sum2[j & 3] = f2_add(sum2[j & 3], f2_pack(p0, p1));
       pk[j] = F16 ? pack_f16x2(p0, p1) : pack_bf16x2(p0, p1);
     }
-    tmem_st16(p_addr + k * 16, pk);
+    tmem_st_cols(p_addr + k * W, pk);
+    if (k + 1 < kPParts) {   // a part of P: O += P V may run its next k-steps
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&part_ready[k]);
+    }
   }
   float a0, a1;
   f2_unpack(f2_add(f2_add(sum2[0], sum2[1]), f2_add(sum2[2], sum2[3])), a0, a1);
   return a0 + a1;
 }
 
-// FP8 query tile -> shared memory as F16 (exact), same K-major swizzled layout as the BF16 tile.
-__device__ __forceinline__ void load_q_tile_f16(uint8_t* sQ, const uint8_t* __restrict__ q, const SegInfo& sg,
-                                                const DevParams& P, int t, int nthr) {
-  const int g = P.group;
-  constexpr int BATCH = 8;
-  for (int i0 = t; i0 < kTileRows * 16; i0 += nthr * BATCH) {
-    uint2 v[BATCH];
-#pragma unroll
-    for (int u = 0; u < BATCH; ++u) {
-      const int i = i0 + u * nthr;
-      const int row = i >> 4, ch = i & 15;   // 16 chunks of 8 elements per row
-      v[u] = make_uint2(0, 0);
-      if (i < kTileRows * 16 && row < sg.nrows) {
-        const int r = sg.r0 + row;
-        const size_t tok = (size_t)sg.q_tok0 + r / g;
-        const size_t head = (size_t)sg.h * g + r % g;
-        v[u] = __ldg(reinterpret_cast<const uint2*>(q + (tok * P.num_q_heads + head) * kHeadDim + ch * 8));
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < BATCH; ++u) {
-      const int i = i0 + u * nthr;
-      const int row = i >> 4, ch = i & 15;
-      if (i < kTileRows * 16) {
-        const uint4 o = make_uint4(e4m3x2_to_f16x2(v[u].x), e4m3x2_to_f16x2(v[u].x >> 16),
-                                   e4m3x2_to_f16x2(v[u].y), e4m3x2_to_f16x2(v[u].y >> 16));
-        *reinterpret_cast<uint4*>(sQ + (ch >> 3) * 16384 + sw128_offset(row, ch & 7)) = o;
-      }
-    }
-  }
-}
-
+// map_kbar / map_kbar_lo: pooled keys of the correction chunks -- BF16: one BF16 array (map_kbar_lo unused);
+// FP8: the e4m3 hi and lo arrays.  map_vbar: pooled values, 16-bit.
 template <bool FP8>
-__global__ void __launch_bounds__(AttnCfg<FP8>::kThreads, 1)
+__global__ void __launch_bounds__(AttnCfg<FP8>::kThreads, AttnCfg<FP8>::kCtasPerSm)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
-                   const __grid_constant__ CUtensorMap map_kbar, const __grid_constant__ CUtensorMap map_vbar,
-                   AttnArgs A, DevParams P) {
-  constexpr int kNQ = AttnCfg<FP8>::kNQ, kNK = AttnCfg<FP8>::kNK, kNV = AttnCfg<FP8>::kNV, kNRaw = AttnCfg<FP8>::kNRaw;
-  constexpr int kAttnThreads = AttnCfg<FP8>::kThreads;
+                    const __grid_constant__ CUtensorMap map_kbar, const __grid_constant__ CUtensorMap map_kbar_lo,
+                    const __grid_constant__ CUtensorMap map_vbar, AttnArgs A, DevParams P) {
+  constexpr int kSetupThreads = 64;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem;
-  uint8_t* sK = smem + kNQ * kTileBytes;
-  uint8_t* sV = sK + kNK * kTileBytes;
-  uint8_t* sRaw = sV + kNV * kTileBytes;                          // FP8 only: raw tile ring
-  float* sX = reinterpret_cast<float*>(sRaw + kNRaw * kRawBytes);  // [2 parity][kWG][128] row-max exchange, then the same for row sums
+  uint8_t* sQ = smem;                                  // 32 KB (BF16) / 16 KB (raw e4m3)
+  uint8_t* sK = smem + (FP8 ? kRawBytes : kTileBytes); // 32 KB
+  uint8_t* sV = sK + kTileBytes;                       // 32 KB, 16-bit
+  uint8_t* sVraw = sV + kTileBytes;                    // FP8 only: 16 KB raw e4m3 V tile
+  (void)sVraw;
 
   __shared__ TileInfo info[2];
-  __shared__ uint32_t sel_bits[2][kMaxBlocks / 32];
-  __shared__ uint64_t info_full[2], info_empty[2], q_full[2], q_empty[2], tile_done;
-  // One tcgen05.commit costs the issuing thread ~70 cycles, so barriers that would be signalled by the same
-  // commit are merged: s_full[a] also releases K stage a (k_empty), v_empty[b] also says that O += P V of an
-  // iteration with parity b has completed (what the lazy rescale waits for).
-  static_assert(kNK == 2 && kNV == 2, "merged barriers assume two K stages and two V stages");
-  __shared__ uint64_t k_full[kNK], v_full[kNV], v_empty[kNV];
-  __shared__ uint64_t s_full[2], p_ready[2];
-  uint64_t* const k_empty = s_full;
-  __shared__ uint64_t raw_full[kNRaw > 0 ? kNRaw : 1], raw_empty[kNRaw > 0 ? kNRaw : 1];
+  __shared__ uint32_t sel_bits[kMaxBlocks / 32];
+  __shared__ uint64_t info_full[2], info_empty[2], q_full, q_empty;
+  // Every barrier below completes exactly once per iteration; with G the iteration's index counted over the
+  // whole kernel, the phase that belongs to iteration G has parity G & 1.
+  __shared__ uint64_t k_full, v_full;
+  __shared__ uint64_t s_done;    // S = Q K^T (G) has completed: the logits are in TMEM, the K stage is free --
+                                 // and, MMAs completing in issue order, O += P V (G-1) is in O
+  __shared__ uint64_t pv_done[2];  // [G & 1], phase (G >> 1) & 1: O += P V (G) has completed -- the V stage is free,
+                                   // O holds iteration G.  Two barriers so that a waiter may be two iterations
+                                   // behind the issuer without mistaking one phase for another.
+  __shared__ uint64_t vraw_full, vraw_empty;   // FP8: the raw V tile has landed / has been widened
+  __shared__ uint64_t p_ready[kPParts];   // slice q (128 / kPParts probabilities of every row) of P (G) is in TMEM
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
 
@@ -232,23 +206,26 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     abort_flag = 0;
     for (int i = 0; i < 2; ++i) {
       mbar_init(&info_full[i], 1);
-      mbar_init(&info_empty[i], 2 + 128 * kWG + (FP8 ? 1 : 0));
-      mbar_init(&s_full[i], 1);
-      mbar_init(&p_ready[i], 128 * kWG);
+      mbar_init(&info_empty[i], 2 + 128);   // producer, issuer, softmax threads
     }
-    for (int i = 0; i < 2; ++i) { mbar_init(&q_full[i], 64); mbar_init(&q_empty[i], 1); }
-    mbar_init(&tile_done, 1);
-    for (int i = 0; i < kNK; ++i) mbar_init(&k_full[i], 1);
-    for (int i = 0; i < kNV; ++i) { mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); }
-    for (int i = 0; i < kNRaw; ++i) { mbar_init(&raw_full[i], 1); mbar_init(&raw_empty[i], 1); }
+    mbar_init(&q_full, kSetupThreads);
+    mbar_init(&vraw_full, 1);
+    mbar_init(&vraw_empty, 1);
+    mbar_init(&q_empty, 1);
+    mbar_init(&k_full, 1);
+    mbar_init(&v_full, 1);
+    mbar_init(&s_done, 1);
+    mbar_init(&pv_done[0], 1);
+    mbar_init(&pv_done[1], 1);
+    for (int i = 0; i < kPParts; ++i) mbar_init(&p_ready[i], 128);
     fence_barrier_init();
   }
-  // K / V rings start zeroed: rows of pages past the end of a sequence are never loaded, and whatever sits
+  // K / V stages start zeroed: rows of pages past the end of a sequence are never loaded, and whatever sits
   // there is multiplied by probabilities that are exactly zero, so it must be finite.
-  for (int i = tid; i < ((kNK + kNV) * kTileBytes + kNRaw * kRawBytes) / 16; i += kAttnThreads)
+  for (int i = tid; i < (2 * kTileBytes + (FP8 ? kRawBytes : 0)) / 16; i += AttnCfg<FP8>::kThreads)
     reinterpret_cast<uint4*>(sK)[i] = make_uint4(0, 0, 0, 0);
-  if (warp == kSW + 1) {
-    tmem_alloc(&tmem_base_s, 512);
+  if (warp == 5) {
+    tmem_alloc(&tmem_base_s, 256);
     tmem_relinquish();
   }
   fence_proxy_async();
@@ -258,46 +235,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
   const uint32_t tmem = tmem_base_s;
   const int g = P.group;
 
-  if (FP8 && warp >= kSW + 4) {
-    // =============================== FP8 -> F16 widening warpgroup ===============================
+  // O += P V (G) has completed.  Safe for a waiter that is at most two iterations behind the issuer.
+  auto wait_pv = [&](uint32_t G, int where) { mbar_wait(&pv_done[G & 1], (G >> 1) & 1, ctx, where); };
+
+  if (warp >= 6) {
+    // =============================== unit set-up + Q staging ===============================
     setmaxnreg_dec<AttnCfg<FP8>::kRegsService>();
-    if constexpr (FP8) {
-      const int t128 = tid - 32 * (kSW + 4);
-      uint32_t kc = 0, vc = 0, rc = 0;
-      for (int it = 0;; ++it) {
-        const int slot = it & 1;
-        mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 601);
-        const TileInfo& ti = info[slot];
-        if (!ti.valid) break;
-        const int T = ti.T, n_it = T + ti.nchunk;
-        for (int i = 0; i < n_it; ++i, ++kc, ++vc) {
-          if (i >= T) continue;   // correction chunks arrive as F16 straight into the K / V rings
-#pragma unroll
-          for (int kv = 0; kv < 2; ++kv, ++rc) {
-            const int rs = rc % kNRaw;
-            const int ds = kv ? (int)(vc % kNV) : (int)(kc % kNK);
-            const uint32_t dc = kv ? vc : kc;
-            const int dn = kv ? kNV : kNK;
-            uint64_t* d_empty = kv ? &v_empty[ds] : &k_empty[ds];
-            uint64_t* d_full = kv ? &v_full[ds] : &k_full[ds];
-            if (dc >= (uint32_t)dn) mbar_wait(d_empty, ((dc / dn) - 1) & 1, ctx, 602);
-            mbar_wait(&raw_full[rs], (rc / kNRaw) & 1, ctx, 603);
-            widen_tile_f16(sRaw + rs * kRawBytes, (kv ? sV : sK) + ds * kTileBytes, t128, 128);
-            fence_proxy_async();
-            named_bar_sync(3, 128);
-            if (t128 == 0) {
-              mbar_arrive(&raw_empty[rs]);
-              mbar_arrive(d_full);
-            }
-          }
-        }
-        if (t128 == 0) mbar_arrive(&info_empty[slot]);
-      }
-    }
-  } else if (warp >= kSW + 2) {
-    // =============================== tile set-up + Q staging ===============================
-    setmaxnreg_dec<AttnCfg<FP8>::kRegsService>();
-    const int t64 = tid - 32 * (kSW + 2);
+    const int t64 = tid - 32 * 6;
     for (int it = 0;; ++it) {
       const int slot = it & 1;
       if (it >= 2) mbar_wait(&info_empty[slot], ((it >> 1) - 1) & 1, ctx, 201);
@@ -320,7 +264,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           ti.valid = 0;
         }
       }
-      named_bar_sync(2, 64);
+      named_bar_sync(2, kSetupThreads);
       const bool valid = ti.valid != 0;
       if (valid && !ti.dense) {
         const SegInfo& sg = ti.sg;
@@ -329,29 +273,29 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         const int nwords = (sg.J_lo + 31) >> 5;
         const bool corr = P.use_correction != 0;
         if (corr)
-          for (int w = t64; w < nwords; w += 64) sel_bits[slot][w] = 0u;
-        named_bar_sync(2, 64);
+          for (int w = t64; w < nwords; w += kSetupThreads) sel_bits[w] = 0u;
+        named_bar_sync(2, kSetupThreads);
         bool bad = false;
-        for (int k = t64; k < T; k += 64) {
+        for (int k = t64; k < T; k += kSetupThreads) {
           const int J = list[k];
           if (J < 0 || J > sg.J_hi || (k > 0 && list[k - 1] >= J)) bad = true;
-          if (corr && J >= 0 && J < sg.J_lo) atomicOr(&sel_bits[slot][J >> 5], 1u << (J & 31));
+          if (corr && J >= 0 && J < sg.J_lo) atomicOr(&sel_bits[J >> 5], 1u << (J & 31));
         }
         if (bad) atomicOr(A.status + ST_BAD_LIST, 1);
-        named_bar_sync(2, 64);
+        named_bar_sync(2, kSetupThreads);
         if (corr) {
           const int nch = (sg.J_lo + 127) >> 7;
-          for (int c = t64; c < nch; c += 64) {
+          for (int c = t64; c < nch; c += kSetupThreads) {
 #pragma unroll
             for (int w = 0; w < 4; ++w) {
               const int first = c * 128 + w * 32;
               uint32_t validm = 0u;
               if (first + 32 <= sg.J_lo) validm = 0xffffffffu;
               else if (first < sg.J_lo) validm = (1u << (sg.J_lo - first)) - 1u;
-              ti.todo[c][w] = (first < sg.J_lo ? ~sel_bits[slot][first >> 5] : 0u) & validm;
+              ti.todo[c][w] = (first < sg.J_lo ? ~sel_bits[first >> 5] : 0u) & validm;
             }
           }
-          named_bar_sync(2, 64);
+          named_bar_sync(2, kSetupThreads);
           if (t64 == 0) {
             int n = 0;
             for (int c = 0; c < nch; ++c)
@@ -360,18 +304,20 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           }
         }
       }
-      named_bar_sync(2, 64);
+      named_bar_sync(2, kSetupThreads);
       if (t64 == 0) mbar_arrive(&info_full[slot]);
       if (!valid) break;
-      // Q tile: wait until every S = Q K^T of the unit that last used this buffer has completed, then overwrite
-      const int qb = it % kNQ;
-      if (it >= kNQ) mbar_wait(&q_empty[qb], ((it / kNQ) - 1) & 1, ctx, 202);
-      if constexpr (FP8) load_q_tile_f16(sQ + qb * kTileBytes, A.q, ti.sg, P, t64, 64);
-      else load_q_tile_async(sQ + qb * kTileBytes, A.q, ti.sg, P, t64, 64);
+      // Q tile: wait until every S = Q K^T of the previous unit has completed, then overwrite
+      if (it >= 1) mbar_wait(&q_empty, (it - 1) & 1, ctx, 202);
+      if constexpr (FP8) {
+        load_q_raw_async(sQ, A.q, ti.sg, P, t64, kSetupThreads);
+        cp_async_wait_all();
+      }
+      else load_q_tile_async(sQ, A.q, ti.sg, P, t64, kSetupThreads);
       fence_proxy_async();
-      mbar_arrive(&q_full[qb]);
+      mbar_arrive(&q_full);
     }
-  } else if (warp == kSW) {
+  } else if (warp == 4) {
     // =============================== TMA producer ===============================
     setmaxnreg_dec<AttnCfg<FP8>::kRegsService>();
     if (lane == 0) {
@@ -380,7 +326,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       tma_prefetch_desc(&map_kbar);
       tma_prefetch_desc(&map_vbar);
     }
-    uint32_t kc = 0, vc = 0, rc = 0;
+    uint32_t G = 0, rc = 0;
     (void)rc;
     const uint64_t keep = l2_policy_evict_last();   // K / V pages and pooled means: shared by many tiles
     const int ppb = P.pages_per_block, psz = P.page_size;
@@ -408,208 +354,209 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         return pid;
       };
       int pid_next = fetch_pid(0);
-      for (int i = 0; i < n_it; ++i) {
-        const int ks = kc % kNK, vs = vc % kNV;
-        uint8_t* dK = sK + ks * kTileBytes;
-        uint8_t* dV = sV + vs * kTileBytes;
+      for (int i = 0; i < n_it; ++i, ++G) {
         const int pid = pid_next;
         pid_next = fetch_pid(i + 1);
+        if (G >= 1) mbar_wait(&s_done, (G - 1) & 1, ctx, 302);   // K stage free
         if (i < T) {
           const int nvalid = __popc(__ballot_sync(0xffffffffu, pid >= 0));
           if constexpr (FP8) {
-            // raw e4m3 tiles (128 bytes per token row) into the raw ring; the widening warpgroup fills the K / V rings
-            const uint32_t rbytes = (uint32_t)nvalid * psz * 128u;
-#pragma unroll
-            for (int kv = 0; kv < 2; ++kv, ++rc) {
-              const int rs = rc % kNRaw;
-              if (rc >= (uint32_t)kNRaw) mbar_wait(&raw_empty[rs], ((rc / kNRaw) - 1) & 1, ctx, 306);
-              if (lane == 0) mbar_arrive_expect_tx(&raw_full[rs], rbytes);
-              __syncwarp();
-              if (pid >= 0)
-                tma_load_3d_hint(sRaw + rs * kRawBytes + lane * psz * 128, kv ? &map_v : &map_k, &raw_full[rs], 0, sg.h,
-                            pid * psz, keep);
+            // raw e4m3 tiles, 128 bytes per token row: K straight into the K stage (the MMA reads it as it
+            // lands), V into the raw slot for the widening warp
+            const uint32_t bytes = (uint32_t)nvalid * psz * 128u;
+            if (lane == 0) mbar_arrive_expect_tx(&k_full, bytes);
+            __syncwarp();
+            if (pid >= 0) tma_load_3d_hint(sK + lane * psz * 128, &map_k, &k_full, 0, sg.h, pid * psz, keep);
+            if (rc >= 1) mbar_wait(&vraw_empty, (rc - 1) & 1, ctx, 306);
+            if (lane == 0) mbar_arrive_expect_tx(&vraw_full, bytes);
+            __syncwarp();
+            if (pid >= 0) tma_load_3d_hint(sVraw + lane * psz * 128, &map_v, &vraw_full, 0, sg.h, pid * psz, keep);
+            ++rc;
+          } else {
+            const uint32_t bytes = (uint32_t)nvalid * psz * 256u;
+            if (lane == 0) mbar_arrive_expect_tx(&k_full, bytes);
+            __syncwarp();
+            if (pid >= 0) {
+              tma_load_3d_hint(sK + lane * psz * 128, &map_k, &k_full, 0, sg.h, pid * psz, keep);
+              tma_load_3d_hint(sK + 16384 + lane * psz * 128, &map_k, &k_full, 64, sg.h, pid * psz, keep);
             }
-            ++kc;
-            ++vc;
-            continue;
-          }
-          const uint32_t bytes = (uint32_t)nvalid * psz * 256u;
-          if (kc >= kNK) mbar_wait(&k_empty[ks], ((kc / kNK) - 1) & 1, ctx, 302);
-          if (lane == 0) mbar_arrive_expect_tx(&k_full[ks], bytes);
-          __syncwarp();
-          if (pid >= 0) {
-            tma_load_3d_hint(dK + lane * psz * 128, &map_k, &k_full[ks], 0, sg.h, pid * psz, keep);
-            tma_load_3d_hint(dK + 16384 + lane * psz * 128, &map_k, &k_full[ks], 64, sg.h, pid * psz, keep);
-          }
-          if (vc >= kNV) mbar_wait(&v_empty[vs], ((vc / kNV) - 1) & 1, ctx, 303);
-          if (lane == 0) mbar_arrive_expect_tx(&v_full[vs], bytes);
-          __syncwarp();
-          if (pid >= 0) {
-            tma_load_3d_hint(dV + lane * psz * 128, &map_v, &v_full[vs], 0, sg.h, pid * psz, keep);
-            tma_load_3d_hint(dV + 16384 + lane * psz * 128, &map_v, &v_full[vs], 64, sg.h, pid * psz, keep);
+            if (G >= 1) wait_pv(G - 1, 303);  // V stage free
+            if (lane == 0) mbar_arrive_expect_tx(&v_full, bytes);
+            __syncwarp();
+            if (pid >= 0) {
+              tma_load_3d_hint(sV + lane * psz * 128, &map_v, &v_full, 0, sg.h, pid * psz, keep);
+              tma_load_3d_hint(sV + 16384 + lane * psz * 128, &map_v, &v_full, 64, sg.h, pid * psz, keep);
+            }
           }
         } else {
           const int row0 = sg.blk_off + ti.chunk_id[i - T] * 128;
-          if (kc >= kNK) mbar_wait(&k_empty[ks], ((kc / kNK) - 1) & 1, ctx, 304);
           if (lane == 0) {
-            mbar_arrive_expect_tx(&k_full[ks], kTileBytes);
-            tma_load_3d_hint(dK, &map_kbar, &k_full[ks], 0, sg.h, row0, keep);
-            tma_load_3d_hint(dK + 16384, &map_kbar, &k_full[ks], 64, sg.h, row0, keep);
+            mbar_arrive_expect_tx(&k_full, kTileBytes);
+            if constexpr (FP8) {   // e4m3 hi | lo, 16 KB each
+              tma_load_3d_hint(sK, &map_kbar, &k_full, 0, sg.h, row0, keep);
+              tma_load_3d_hint(sK + 16384, &map_kbar_lo, &k_full, 0, sg.h, row0, keep);
+            } else {
+              tma_load_3d_hint(sK, &map_kbar, &k_full, 0, sg.h, row0, keep);
+              tma_load_3d_hint(sK + 16384, &map_kbar, &k_full, 64, sg.h, row0, keep);
+            }
           }
-          if (vc >= kNV) mbar_wait(&v_empty[vs], ((vc / kNV) - 1) & 1, ctx, 305);
+          if (G >= 1) wait_pv(G - 1, 305);    // V stage free
           if (lane == 0) {
-            mbar_arrive_expect_tx(&v_full[vs], kTileBytes);
-            tma_load_3d_hint(dV, &map_vbar, &v_full[vs], 0, sg.h, row0, keep);
-            tma_load_3d_hint(dV + 16384, &map_vbar, &v_full[vs], 64, sg.h, row0, keep);
+            mbar_arrive_expect_tx(&v_full, kTileBytes);
+            tma_load_3d_hint(sV, &map_vbar, &v_full, 0, sg.h, row0, keep);
+            tma_load_3d_hint(sV + 16384, &map_vbar, &v_full, 64, sg.h, row0, keep);
           }
           __syncwarp();
         }
-        ++kc;
-        ++vc;
       }
       if (lane == 0) mbar_arrive(&info_empty[slot]);
     }
-  } else if (warp == kSW + 1) {
+  } else if (warp == 5) {
     // =============================== UMMA issuer ===============================
     setmaxnreg_dec<AttnCfg<FP8>::kRegsService>();
     if (lane == 0) {
-      constexpr int kFmt = AttnCfg<FP8>::kFmt;
-      constexpr uint32_t idesc_qk = make_idesc(128, 128, kFmt, kFmt, 0, 0);
+      constexpr int kFmt = FP8 ? 0 : 1;   // kind::f16 operand format of O += P V: 0 = F16, 1 = BF16
+      constexpr uint32_t idesc_qk = FP8 ? make_idesc(128, 128, 0, 0, 0, 0)    // kind::f8f6f4, E4M3 x E4M3
+                                        : make_idesc(128, 128, 1, 1, 0, 0);
       constexpr uint32_t idesc_pv = make_idesc(128, 128, kFmt, kFmt, 0, 1);
-      uint32_t kc = 0, vc = 0, pc0 = 0, pc1 = 0;
-      auto issue_pv = [&](int j) {
-        const int b = vc & 1;   // P buffer / V stage: parity of the iteration counted over the whole kernel
-        if (b) { mbar_wait(&p_ready[1], pc1 & 1, ctx, 401); ++pc1; }
-        else { mbar_wait(&p_ready[0], pc0 & 1, ctx, 401); ++pc0; }
-        const int vs = vc % kNV;
-        mbar_wait(&v_full[vs], (vc / kNV) & 1, ctx, 402);
-        tc_fence_after();
-        const uint32_t v_addr = smem_u32(sV + vs * kTileBytes);
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint64_t bd = make_smem_desc_sw128(v_addr + ks * 2048, 16384, 1024);
-          umma_f16_ts(tmem + 256, tmem + 384 + b * 64 + ks * 8, bd, idesc_pv, (j > 0) || ks > 0);
-        }
-        umma_commit(&v_empty[vs]);   // V stage vs (== iteration parity) is free and O holds this iteration
-        ++vc;
-      };
+      const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+      uint32_t G = 0;
       for (int it = 0;; ++it) {
         const int slot = it & 1;
         mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 403);
         const TileInfo& ti = info[slot];
         if (!ti.valid) break;
-        const int n_it = ti.T + ti.nchunk;
-        const int qb = it % kNQ;
-        mbar_wait(&q_full[qb], (it / kNQ) & 1, ctx, 404);
-        const uint32_t q_addr = smem_u32(sQ + qb * kTileBytes);
-        for (int i = 0; i < n_it; ++i) {
-          const int ks_ = kc % kNK;
-          const int a = ks_;   // S buffer = K stage = parity of the iteration counted over the whole kernel
-          mbar_wait(&k_full[ks_], (kc / kNK) & 1, ctx, 405);
+        const int T = ti.T, n_it = T + ti.nchunk;
+        (void)T;
+        mbar_wait(&q_full, it & 1, ctx, 404);
+        for (int i = 0; i < n_it; ++i, ++G) {
+          // S = Q K^T (G).  The S columns are free: O += P V (G-1), which read P out of them, was issued before.
+          mbar_wait(&k_full, G & 1, ctx, 405);
           tc_fence_after();
-          const uint32_t k_addr = smem_u32(sK + ks_ * kTileBytes);
-          // S_a is free: the softmax of iteration i-2 signalled p_ready[a] (waited for in issue_pv(i-2))
+          if constexpr (FP8) {
+            // raw e4m3 operands, 32 elements (= 32 bytes of the swizzled row) per MMA; a correction chunk adds
+            // the lo part of the pooled keys on top of the hi part
+            const int parts = i < T ? 1 : 2;
+            for (int part = 0; part < parts; ++part) {
 #pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
-            const uint64_t ad = make_smem_desc_sw128(q_addr + off, 16, 1024);
-            const uint64_t bd = make_smem_desc_sw128(k_addr + off, 16, 1024);
-            umma_f16_ss(tmem + a * 128, ad, bd, idesc_qk, ks > 0);
+              for (int ks = 0; ks < 4; ++ks) {
+                const uint64_t ad = make_smem_desc_sw128(q_addr + ks * 32, 16, 1024);
+                const uint64_t bd = make_smem_desc_sw128(k_addr + part * 16384 + ks * 32, 16, 1024);
+                umma_f8_ss(tmem, ad, bd, idesc_qk, (part > 0) || ks > 0);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+              const uint64_t ad = make_smem_desc_sw128(q_addr + off, 16, 1024);
+              const uint64_t bd = make_smem_desc_sw128(k_addr + off, 16, 1024);
+              umma_f16_ss(tmem, ad, bd, idesc_qk, ks > 0);
+            }
           }
-          umma_commit(&s_full[a]);   // S_a is ready and K stage ks_ (== a) is free
-          ++kc;
-          if (i == n_it - 1) umma_commit(&q_empty[qb]);
-          if (i >= 1) issue_pv(i - 1);
+          umma_commit(&s_done);
+          if (i == n_it - 1) umma_commit(&q_empty);
+          // O += P V (G)
+          mbar_wait(&v_full, G & 1, ctx, 402);
+#pragma unroll
+          for (int h = 0; h < kPParts; ++h) {   // as each slice of P arrives
+            mbar_wait(&p_ready[h], G & 1, ctx, 401);
+            tc_fence_after();
+#pragma unroll
+            for (int ks = (8 / kPParts) * h; ks < (8 / kPParts) * (h + 1); ++ks) {
+              const uint64_t bd = make_smem_desc_sw128(v_addr + ks * 2048, 16384, 1024);
+              umma_f16_ts(tmem + 128, tmem + ks * 8, bd, idesc_pv, (i > 0) || ks > 0);
+            }
+          }
+          umma_commit(&pv_done[G & 1]);
         }
-        if (n_it >= 1) issue_pv(n_it - 1);
-        else umma_commit(&q_empty[qb]);  // empty list: nothing read Q, release it at once
-        umma_commit(&tile_done);
+        if (n_it == 0) umma_commit(&q_empty);  // empty list: nothing read Q, release it at once
         mbar_arrive(&info_empty[slot]);
       }
     }
   } else {
-    // =============================== softmax warpgroups + epilogue ===============================
+    // =============================== softmax warpgroup + epilogue ===============================
     setmaxnreg_inc<AttnCfg<FP8>::kRegsSoftmax>();
-    const int wg = warp >> 2;
-    const int row = (warp & 3) * 32 + lane;
-    const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
-    const uint32_t o_addr = lane_base + 256 + wg * kCW;   // this thread's kCW columns of O
-    uint32_t sc0 = 0, sc1 = 0;   // completed uses of S0 / S1 (phases of s_full)
-    uint32_t pv_base = 0;        // iterations (= UMMA groups O += P V = V stage uses) before this tile
+    const int row = warp * 32 + lane;
+    const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t s_addr = lane_base;         // S; P overwrites its first 64 columns
+    const uint32_t o_addr = lane_base + 128;
+    uint32_t G = 0, rc = 0;   // rc: exact iterations so far (uses of the raw V slot)
+    (void)rc;
     const uint64_t stream_pol = l2_policy_evict_first();   // outputs are written once and not read here
     for (int it = 0;; ++it) {
       const int slot = it & 1;
       mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 501);
       const TileInfo& ti = info[slot];
       if (!ti.valid) break;
-      const SegInfo sg = ti.sg;
       const int T = ti.T, n_it = T + ti.nchunk;
-      const int32_t* list = A.blk_idx + sg.off;
-      const int r = sg.r0 + row;
-      const int pos = sg.pre + r / g;
-      // logit multipliers in log2 units.  FP8 (Eq. 15): the MMAs see raw e4m3 values, so exact blocks carry
-      // q_scale * k_scale and pooled chunks (kbar is stored de-scaled) carry q_scale only.
-      float cs_exact = P.scale_log2, cs_chunk = P.scale_log2, out_scale = 1.0f;
+      const bool dense = ti.dense != 0;
+      const int J_hi = ti.sg.J_hi, J_lo = ti.sg.J_lo;
+      const int32_t* list = A.blk_idx + ti.sg.off;
+      const int r = ti.sg.r0 + row;
+      const int pos = ti.sg.pre + r / g;
+      // logit multiplier in log2 units.  FP8 (Eq. 15): the MMAs see raw e4m3 values (pooled keys included), so
+      // every logit of a row carries q_scale * k_scale; the output carries v_scale.
+      float cs_all = P.scale_log2, out_scale = 1.0f;
       if constexpr (FP8) {
-        const float qs = A.q_scale[sg.h * g + r % g];
-        cs_chunk *= qs;
-        cs_exact *= qs * A.k_scale[sg.h];
-        out_scale = A.v_scale[sg.h];
+        cs_all *= A.q_scale[ti.sg.h * g + r % g] * A.k_scale[ti.sg.h];
+        out_scale = A.v_scale[ti.sg.h];
       }
       float m = -INFINITY, l = 0.f;
       // block id of the next exact iteration, fetched one iteration ahead
-      int J_next = (!ti.dense && T > 0) ? list[T - 1] : 0;
-      for (int i = 0; i < n_it; ++i) {
-        const int a = (pv_base + i) & 1;   // S / P buffer: parity of the iteration counted over the whole kernel
-        const uint32_t s_addr = lane_base + a * 128 + wg * kCW;
-        const uint32_t p_addr = lane_base + 384 + a * 64 + wg * (kCW / 2);
+      int J_next = (!dense && T > 0) ? list[T - 1] : 0;
+      for (int i = 0; i < n_it; ++i, ++G) {
         // iteration kind and masks
         bool need_mask = false;
         int tok_lim = 1 << 30;     // exact block: columns j with j <= tok_lim are visible
-        uint32_t cm[kCW / 32];
-#pragma unroll
-        for (int w = 0; w < kCW / 32; ++w) cm[w] = 0xffffffffu;
-        float shift = 0.f, cs = cs_exact;
+        uint32_t cm0 = 0xffffffffu, cm1 = 0xffffffffu, cm2 = 0xffffffffu, cm3 = 0xffffffffu;
+        float shift = 0.f;
         if (i < T) {
-          int J = ti.dense ? sg.J_hi - i : J_next;
-          if (!ti.dense && i + 1 < T) J_next = list[T - 2 - i];
-          J = max(0, min(J, sg.J_hi));
-          need_mask = J >= sg.J_lo;
+          int J = dense ? J_hi - i : J_next;
+          if (!dense && i + 1 < T) J_next = list[T - 2 - i];
+          J = max(0, min(J, J_hi));
+          need_mask = J >= J_lo;
           tok_lim = pos - J * kBlock;
         } else {
           const int c = ti.chunk_id[i - T];
-#pragma unroll
-          for (int w = 0; w < kCW / 32; ++w) cm[w] = ti.todo[c][wg * (kCW / 32) + w];
+          cm0 = ti.todo[c][0];
+          cm1 = ti.todo[c][1];
+          cm2 = ti.todo[c][2];
+          cm3 = ti.todo[c][3];
           shift = 7.0f;  // log2(128): one pooled row stands for a full block (Eq. 6)
-          cs = cs_chunk;
           need_mask = true;
         }
-        if (a) { mbar_wait(&s_full[1], sc1 & 1, ctx, 502); ++sc1; }
-        else { mbar_wait(&s_full[0], sc0 & 1, ctx, 502); ++sc0; }
+        if constexpr (FP8) {
+          // Exact iteration: widen this iteration's raw e4m3 V tile (exactly) into the F16 V stage before looking
+          // at the logits.  128 threads take ~900 cycles (the copy is bound by shared-memory bandwidth next to the
+          // other CTA's MMAs); one or two dedicated warps were slower than the time they have, between
+          // O += P V (G-1) freeing the stage and the first slice of P (G) needing it.
+          if (i < T) {
+            mbar_wait(&vraw_full, rc & 1, ctx, 603);
+            if (G >= 1) wait_pv(G - 1, 602);
+            widen_tile_f16(sVraw, sV, tid, 128);
+            fence_proxy_async();
+            named_bar_sync(1, 128);
+            if (tid == 0) {
+              mbar_arrive(&vraw_empty);
+              mbar_arrive(&v_full);
+            }
+            ++rc;
+          }
+        }
+        mbar_wait(&s_done, G & 1, ctx, 502);
         tc_fence_after();
-        if (need_mask) mask_cols(s_addr, wg * kCW, tok_lim, cm);
-        // row maximum over all 128 columns: own half, then the other warpgroup's through shared memory
-        uint32_t sv[kCW];
-        float mx = cols_row_max(s_addr, sv);
-        float* xch = sX + (i & 1) * (kWG * 128);
-        xch[wg * 128 + row] = mx;
-        named_bar_sync(1, 128 * kWG);
-#pragma unroll
-        for (int w = 1; w < kWG; ++w) mx = fmaxf(mx, xch[((wg + w) % kWG) * 128 + row]);
-        mx = fmaf(mx, cs, shift);  // cs > 0: scaling commutes with the maximum
+        if (need_mask) mask_row(s_addr, tok_lim, cm0, cm1, cm2, cm3);
+        uint32_t x[128];
+        const float mx = fmaf(row_load_max(s_addr, x), cs_all, shift);  // cs > 0: scaling commutes with the maximum
         const float m_new = fmaxf(m, mx);
-        // lazy rescale: only when some row of the warp moved its maximum by more than 2^8.  Both warpgroups
-        // hold the same rows in the same warps and the same m, so they take the same decision.
-        const bool need = m_new > m + 8.0f;
-        if (__any_sync(0xffffffffu, need)) {
+        // lazy rescale: only when some row of the warp moved its maximum by more than 2^8.  O is at rest: the
+        // MMAs complete in issue order, so S (G) in TMEM means O += P V (G-1) has been added.
+        if (__any_sync(0xffffffffu, m_new > m + 8.0f)) {
           const float f = (m == -INFINITY) ? 0.f : ex2(m - m_new);
           if (i > 0) {
-            // O must be at rest: wait for O += P V of iteration i-1, the ((pv_base + i - 1) / 2)-th use of V stage
-            // (pv_base + i - 1) % 2 counted over the whole kernel (iterations and V stages advance together)
-            mbar_wait(&v_empty[(pv_base + i - 1) & 1], ((pv_base + i - 1) >> 1) & 1, ctx, 504);
-            tc_fence_after();
-#pragma unroll
-            for (int k = 0; k < kCW / 32; ++k) {
+#pragma unroll 1
+            for (int k = 0; k < 4; ++k) {
               uint32_t rr[32];
               tmem_ld32(o_addr + k * 32, rr);
               tmem_wait_ld();
@@ -623,29 +570,25 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         }
         // a row with nothing visible so far has m = -inf and only -inf logits: exponent against 0 -> zeros
         const float neg_m = (m == -INFINITY) ? shift : shift - m;
-        l += cols_row_exp<FP8>(sv, p_addr, cs, neg_m);
+        l += row_exp<FP8>(x, s_addr, cs_all, neg_m, &p_ready[0]);
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&p_ready[a]);
+        mbar_arrive(&p_ready[kPParts - 1]);
       }
-      pv_base += (uint32_t)n_it;
       // ------------------------------ epilogue ------------------------------
-      mbar_wait(&tile_done, it & 1, ctx, 503);
-      tc_fence_after();
-      float* xch = sX + 2 * kWG * 128 + (it & 1) * (kWG * 128);   // by tile parity: no barrier before its next use
-      xch[wg * 128 + row] = l;
-      named_bar_sync(1, 128 * kWG);
-      float L = l;
-#pragma unroll
-      for (int w = 1; w < kWG; ++w) L += xch[((wg + w) % kWG) * 128 + row];
-      const float inv = L > 0.f ? out_scale / L : 0.f;
+      const SegInfo& sg = ti.sg;
+      const float inv = l > 0.f ? out_scale / l : 0.f;
       const bool have_o = n_it >= 1;
       const bool row_ok = row < sg.nrows;
       const size_t tok = (size_t)sg.q_tok0 + r / g;
       const int head = sg.h * g + r % g;
-      __nv_bfloat16* orow = A.out + (tok * P.num_q_heads + head) * kHeadDim + wg * kCW;
-#pragma unroll
-      for (int k = 0; k < kCW / 32; ++k) {
+      __nv_bfloat16* orow = A.out + (tok * P.num_q_heads + head) * kHeadDim;
+      if (have_o) {
+        wait_pv(G - 1, 503);   // O += P V of the unit's last iteration
+        tc_fence_after();
+      }
+#pragma unroll 1
+      for (int k = 0; k < 4; ++k) {
         uint32_t a0[32];
         if (have_o) {
           tmem_ld32(o_addr + k * 32, a0);
@@ -663,8 +606,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           st_global_v8(orow + k * 32 + 16, &o[8], stream_pol);
         }
       }
-      if (wg == 0 && row_ok && A.lse != nullptr)
-        A.lse[(size_t)head * P.total_q + tok] = (m + log2f(L)) * 0.6931471805599453f;
+      if (row_ok && A.lse != nullptr)
+        A.lse[(size_t)head * P.total_q + tok] = (m + log2f(l)) * 0.6931471805599453f;
       tc_fence_before();
       mbar_arrive(&info_empty[slot]);
     }
@@ -673,7 +616,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
   if (abort_flag) __nanosleep(2000000);
   tc_fence_before();
   __syncthreads();
-  if (warp == kSW + 1) tmem_dealloc(tmem, 512);
+  if (warp == 5) tmem_dealloc(tmem, 256);
 }
 
 }  // namespace fp2
