@@ -28,6 +28,12 @@ forms):
   * comparison is ">=": equality selects;
   * LSE is the natural log of the corrected denominator, softmax scale included.
 
+Index export (Algorithm 1 line 5; Sec. 3.3 "Index-Driven Sparse Traversal", Eq. 17; Sec. 4.4
+"Serving Integration"): the block lists as a compact CSR of physical tiles, and the
+page-level table taken from a token-level slot map by striding.  Readings: a logical block
+expands to the physical tiles that hold at least one real token of it (B / tile_tokens of
+them except in a ragged last block); `cu` is the running count in segment order.
+
 Parity pins: every function here is pinned by tests that do not go through this file's
 own formulae (dense limit against a naive loop and torch SDPA, the block-constant closed
 form, brute force on tiny inputs, Eq. 1-3 against Eq. 19-20, invariants).  What is NOT
@@ -368,3 +374,45 @@ def scatter_output(wl: Workload, results, total_q: int):
         O[tok, head] = o
         L[head, tok] = lse
     return O, L
+
+
+# ------------------------------------------------------------------------------------------
+# Index export
+# ------------------------------------------------------------------------------------------
+
+def export_csr(wl: Workload, lists, tile_tokens: int = 64):
+    """Algorithm 1 line 5: (cu, idx) with every listed logical block J of a segment replaced by the
+    physical tiles (tile_tokens tokens each) that intersect its real tokens [J B, min((J+1) B, Lk)).
+    cu: int64 [nseg + 1] (exclusive running count, Eq. 17's cu[g]); idx: int32 ascending per segment."""
+    B = wl.p.block_size
+    cu = [0]
+    idx: List[int] = []
+    for s in wl.segs:
+        Lk = int(wl.lk[s.b])
+        for J in lists[s.seg]:
+            first, last = int(J) * B, min((int(J) + 1) * B, Lk)      # real tokens of the block
+            t = first // tile_tokens
+            while t * tile_tokens < last:
+                idx.append(t)
+                t += 1
+        cu.append(len(idx))
+    return np.asarray(cu, dtype=np.int64), np.asarray(idx, dtype=np.int32)
+
+
+def page_table_from_token_map(token_to_slot: np.ndarray, seqlens_k: Sequence[int], page_size: int,
+                              max_pages: int):
+    """Sec. 4.4: the page-level table is the token-level slot map read every page_size entries.
+    token_to_slot [ns, max_tokens]: global slot of token j of sequence b (Eq. 22's addr(b, j)).
+    Returns (page_table int32 [ns, max_pages] with -1 past the last page, misaligned) where misaligned
+    says some sampled slot was not the first slot of a page."""
+    ns = len(seqlens_k)
+    pt = np.full((ns, max_pages), -1, dtype=np.int32)
+    misaligned = False
+    for b in range(ns):
+        for k in range(max_pages):
+            if k * page_size >= int(seqlens_k[b]):
+                break
+            slot = int(token_to_slot[b, k * page_size])
+            misaligned |= slot % page_size != 0
+            pt[b, k] = slot // page_size
+    return pt, misaligned

@@ -513,3 +513,93 @@ def test_generator_density_matches_forced_fraction_on_config1():
     nsel = sum(len(v[0]) for v in sel.values())
     forced = sum(int(O.forced_mask(s.J_lo, s.J_hi, 128, 256, 512).sum()) for s in wl.segs)
     assert forced == 364 and nsel >= forced and nsel <= 544
+
+
+# ------------------------------------------------------------------------------------------
+# index export (Algorithm 1 line 5; Sec. 4.4): pinned by token coverage, by the paper's
+# "B / 64 physical tiles per logical block" and its index-memory figure, and by the round trip
+# through Eq. 22
+# ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("tile", [16, 32, 64, 128])
+def test_export_csr_covers_exactly_the_listed_tokens(tile):
+    wl, raw = tiny_workload(31, [(500, 100), (129, 0), (64, 0), (333, 300)], Hq=4, Hkv=2, d=8, B=128, M=128, p=16)
+    sel = O.oracle_select(wl)
+    lists = {seg: v[0] for seg, v in sel.items()}
+    cu, idx = O.export_csr(wl, lists, tile)
+    assert cu[0] == 0 and len(cu) == len(wl.segs) + 1 and cu[-1] == len(idx)
+    assert (np.diff(cu) >= 0).all()
+    for s in wl.segs:
+        Lk = int(wl.lk[s.b])
+        tiles = idx[cu[s.seg]:cu[s.seg + 1]]
+        assert (np.diff(tiles) > 0).all()                      # ascending, unique
+        want = np.zeros(Lk, dtype=bool)                        # tokens of the listed blocks, one by one
+        for J in lists[s.seg]:
+            want[J * 128:min((J + 1) * 128, Lk)] = True
+        got = np.zeros(Lk + tile, dtype=bool)
+        for t in tiles:
+            assert t * tile < Lk                               # every tile holds a real token
+            got[t * tile:(t + 1) * tile] = True
+        # a tile may reach past its block only inside the same block's padding (tile <= B divides B)
+        assert (got[:Lk] == want).all()
+
+
+def test_export_csr_two_tiles_per_full_block_and_paper_index_memory():
+    """B / 64 = 2 physical tiles per logical block (Sec. 3.3, implementation details); with every block
+    listed at 128K (32 query heads, 4 KV heads) the index holds 2 x pairs int32 entries, and at the paper's
+    5 % density that is its 6 MB figure."""
+    gold = _golden()
+    p = O.Params(num_q_heads=32, num_kv_heads=4)
+    L = 4096
+
+    class W:   # geometry only: export_csr touches segments and lengths, never the tensors
+        pass
+    wl = W()
+    wl.p, wl.lk = p, np.array([L])
+    wl.segs = O.segments(p, [0, L], [L])
+    lists = {s.seg: np.arange(s.J_hi + 1) for s in wl.segs}
+    cu, idx = O.export_csr(wl, lists, 64)
+    pairs = sum(s.J_hi + 1 for s in wl.segs)
+    assert cu[-1] == 2 * pairs
+    s0 = wl.segs[5]
+    assert list(idx[cu[5]:cu[6]]) == [t for J in range(s0.J_hi + 1) for t in (2 * J, 2 * J + 1)]
+    # scale the count to 128K (pairs grow with L^2) and apply the paper's density
+    pairs_128k = sum(s.J_hi + 1 for s in O.segments(p, [0, 131072], [131072]))
+    mb = 2 * pairs_128k * gold["csr_density_128k"] * 4 / 1e6
+    assert abs(mb - gold["csr_mb_128k"]) / gold["csr_mb_128k"] < 0.2
+
+
+def test_export_csr_ragged_last_block():
+    p = O.Params(num_q_heads=1, num_kv_heads=1)
+
+    class W:
+        pass
+    for Lk, n_last in ((128 + 1, 1), (128 + 64, 1), (128 + 65, 2), (256, 2)):
+        wl = W()
+        wl.p, wl.lk = p, np.array([Lk])
+        wl.segs = O.segments(p, [0, Lk], [Lk])
+        last = wl.segs[-1]
+        cu, idx = O.export_csr(wl, {s.seg: np.arange(s.J_hi + 1) for s in wl.segs}, 64)
+        assert cu[last.seg + 1] - cu[last.seg] == 2 * last.J_hi + n_last
+
+
+def test_page_table_from_token_map_round_trip():
+    """Eq. 22 forwards (slot of every token from the page table), then the strided read backwards."""
+    rng = np.random.default_rng(5)
+    p, lens = 16, [500, 17, 16, 129]
+    need = [-(-L // p) for L in lens]
+    ids = rng.permutation(sum(need) + 5)
+    pt = np.full((len(lens), max(need)), -1, dtype=np.int32)
+    o = 0
+    for b, n in enumerate(need):
+        pt[b, :n] = ids[o:o + n]
+        o += n
+    tok = np.full((len(lens), max(lens)), -7, dtype=np.int32)
+    for b, L in enumerate(lens):
+        for j in range(L):
+            tok[b, j] = pt[b, j // p] * p + j % p            # Eq. 22
+    got, bad = O.page_table_from_token_map(tok, lens, p, pt.shape[1])
+    assert not bad and (got == pt).all()
+    tok[3, 32] += 3                                            # a slot that does not start a page
+    got, bad = O.page_table_from_token_map(tok, lens, p, pt.shape[1])
+    assert bad
