@@ -299,6 +299,14 @@ def main():
                              "sparse_ms_min": float(np.min(att_ms)), "executed_tflops": achieved,
                              "tokens_per_s": case.total_q / (ms_step * 1e-3),
                              "speedup_vs_own_dense": float(np.mean(dense_ms)) / ms_step}
+        # index export of the headline lists (Algorithm 1 line 5): compact CSR of 64-token physical tiles.
+        # Algorithmic bytes: the lists read once (4 B per listed block), two int32 written per block, one
+        # 56-byte segment record and one count read and one cu entry written per segment.
+        exp_ms = timed(lambda: dc.export_csr(64), 5, 3)
+        exp_bytes = sel_pairs * (4 + 8) + dc.plan.num_segments * (56 + 4 + 4)
+        extra["export_csr"] = {"tile_tokens": 64, "entries": int(2 * sel_pairs), "ms": float(np.mean(exp_ms)),
+                               "gbs": exp_bytes / (np.mean(exp_ms) * 1e-3) / 1e9,
+                               "note": "3 launches; includes two torch.empty allocations of the helper"}
         if not args.no_sweep:
             sweep = []
             for target in (0.5, 0.75, 0.9, 0.95, 0.98):

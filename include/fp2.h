@@ -151,6 +151,29 @@ fp2_status fp2_dense_prefill_static(fp2_plan* plan, const void* q, const void* k
                                     const int32_t* seqlens_k, const float* q_scale, const float* k_scale,
                                     const float* v_scale, void* out, float* lse, fp2_stream stream);
 
+/* Index export (Algorithm 1 line 5; Sec. 3.3 "Index-Driven Sparse Traversal", Eq. 17).  Turns the padded lists
+ * (seg_count, blk_idx as fp2_select_blocks writes them or as a caller supplies them) into a compact CSR over
+ * physical tiles of `tile_tokens` tokens (16, 32, 64 or 128; the paper's kernels use 64): every listed logical
+ * block J becomes the tiles J*(128/tile_tokens) ... that hold at least one token of the sequence, ascending.
+ *   out: cu  int32 [num_segments + 1]   cu[g] = first entry of segment g, cu[num_segments] = total entries;
+ *        idx int32 [idx_len]            idx_len must be at least idx_capacity * (128 / tile_tokens).
+ * Segments are in segment order (KV-head-major inside a sequence), i.e. the index is organised per KV head.
+ * Malformed list entries are clamped as in fp2_sparse_prefill and flagged in the status block of `workspace`.
+ * FP2_ERR_UNSUPPORTED if the worst-case entry count does not fit int32, FP2_ERR_CAPACITY if idx_len is too
+ * small.  All pointers device memory; three small kernels on `stream`; nothing is allocated. */
+fp2_status fp2_export_csr(fp2_plan* plan, const int32_t* seg_count, const int32_t* blk_idx, int32_t tile_tokens,
+                          int32_t* cu, int32_t* idx, int64_t idx_len, void* workspace, fp2_stream stream);
+
+/* Page-level table from a token-level slot map (Sec. 4.4 "Serving Integration": the page index is the token-level
+ * mapping read every page_size entries; Eq. 22 is the inverse).  token_to_slot int32 [num_seqs, max_tokens] holds
+ * the global slot (page * page_size + offset) of token j of sequence b; entries past seqlens_k[b] are not read.
+ *   out: page_table int32 [num_seqs, max_pages_per_seq], -1 for pages past the end of a sequence.
+ * A sampled slot that is negative or not the first slot of a page is flagged in the status block
+ * (fp2_read_status returns FP2_ERR_INVALID_ARG).  Device pointers; one kernel on `stream`. */
+fp2_status fp2_page_table_from_token_map(fp2_plan* plan, const int32_t* token_to_slot, int32_t max_tokens,
+                                         const int32_t* seqlens_k, int32_t* page_table, void* workspace,
+                                         fp2_stream stream);
+
 /* Synchronises `stream`, reads the status block of `workspace` and clears it.  Returns FP2_ERR_TIMEOUT if a
  * bounded wait expired, FP2_ERR_INVALID_ARG if a list entry had to be clamped, else FP2_OK.  If
  * h_status_words is not NULL it receives the 8 raw int32 words (host memory). */

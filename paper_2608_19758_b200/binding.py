@@ -18,8 +18,8 @@ STATUS_NAMES = {0: "FP2_OK", 1: "FP2_ERR_INVALID_ARG", 2: "FP2_ERR_UNSUPPORTED",
                 4: "FP2_ERR_CUDA", 5: "FP2_ERR_TIMEOUT"}
 
 EXPORTS = ["fp2_plan_create", "fp2_plan_sizes", "fp2_plan_destroy", "fp2_plan_segment", "fp2_select_blocks",
-           "fp2_sparse_prefill", "fp2_dense_prefill", "fp2_dense_prefill_static", "fp2_read_status", "fp2_last_launch_count",
-           "fp2_status_string"]
+           "fp2_sparse_prefill", "fp2_dense_prefill", "fp2_dense_prefill_static", "fp2_export_csr",
+           "fp2_page_table_from_token_map", "fp2_read_status", "fp2_last_launch_count", "fp2_status_string"]
 
 
 class Fp2Error(RuntimeError):
@@ -74,6 +74,10 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.fp2_dense_prefill_static.argtypes = [C.c_void_p, vp, vp, vp, i32p, i32p, i32p, f32p, f32p, f32p, vp, f32p,
                                              C.c_void_p]
     lib.fp2_dense_prefill_static.restype = C.c_int
+    lib.fp2_export_csr.argtypes = [C.c_void_p, i32p, i32p, C.c_int32, i32p, i32p, C.c_int64, vp, C.c_void_p]
+    lib.fp2_export_csr.restype = C.c_int
+    lib.fp2_page_table_from_token_map.argtypes = [C.c_void_p, i32p, C.c_int32, i32p, i32p, vp, C.c_void_p]
+    lib.fp2_page_table_from_token_map.restype = C.c_int
     lib.fp2_read_status.argtypes = [C.c_void_p, vp, C.POINTER(C.c_int32), C.c_void_p]
     lib.fp2_read_status.restype = C.c_int
     lib.fp2_last_launch_count.argtypes = [C.c_void_p]
@@ -193,6 +197,19 @@ def fp2_dense_prefill_static(plan: Plan, q, k_cache, v_cache, page_table, cu_seq
            "fp2_dense_prefill_static")
 
 
+def fp2_export_csr(plan: Plan, seg_count, blk_idx, tile_tokens: int, cu, idx, workspace, stream=None):
+    """Compact CSR of physical tiles (cu int32 [nseg + 1], idx int32) from the padded block lists."""
+    _check(load().fp2_export_csr(plan.handle, _ptr(seg_count), _ptr(blk_idx), tile_tokens, _ptr(cu), _ptr(idx),
+                                 idx.numel(), _ptr(workspace), _stream(stream)), "fp2_export_csr")
+
+
+def fp2_page_table_from_token_map(plan: Plan, token_to_slot, seqlens_k, page_table, workspace, stream=None):
+    """Page-level table [num_seqs, max_pages_per_seq] from a token-level slot map [num_seqs, max_tokens]."""
+    _check(load().fp2_page_table_from_token_map(plan.handle, _ptr(token_to_slot), token_to_slot.shape[1],
+                                                _ptr(seqlens_k), _ptr(page_table), _ptr(workspace),
+                                                _stream(stream)), "fp2_page_table_from_token_map")
+
+
 def fp2_read_status(plan: Plan, workspace, stream=None, raise_on_error: bool = True):
     words = (C.c_int32 * 8)()
     code = load().fp2_read_status(plan.handle, _ptr(workspace), words, _stream(stream))
@@ -240,6 +257,13 @@ class DeviceCase:
         fp2_dense_prefill(self.plan, self.q, self.k_cache, self.v_cache, self.page_table, self.cu_seqlens_q,
                           self.seqlens_k, self.q_scale, self.k_scale, self.v_scale, self.out, self.lse,
                           self.workspace)
+
+    def export_csr(self, tile_tokens=64):
+        """(cu, idx) device tensors of the lists currently in the buffers."""
+        cu = torch.empty(self.plan.num_segments + 1, dtype=torch.int32, device=self.q.device)
+        idx = torch.empty(max(self.plan.idx_capacity * (128 // tile_tokens), 1), dtype=torch.int32, device=self.q.device)
+        fp2_export_csr(self.plan, self.seg_count, self.blk_idx, tile_tokens, cu, idx, self.workspace)
+        return cu, idx
 
     def status(self, raise_on_error=True):
         return fp2_read_status(self.plan, self.workspace, raise_on_error=raise_on_error)

@@ -14,6 +14,7 @@
 #include "pool_kv.cuh"
 #include "score_select.cuh"
 #include "sparse_attn.cuh"
+#include "index_export.cuh"
 
 using namespace fp2;
 
@@ -498,6 +499,58 @@ extern "C" fp2_status fp2_dense_prefill_static(fp2_plan* pl, const void* q, cons
   // the dense path stages no pooled chunks: the two pooled-mean maps are never dereferenced
   launch_attn(pl, mk, mv, mk, mk, mv, a, st);
   pl->last_launches = 4;
+  return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Index export
+// ------------------------------------------------------------------------------------------------------
+extern "C" fp2_status fp2_export_csr(fp2_plan* pl, const int32_t* seg_count, const int32_t* blk_idx,
+                                     int32_t tile_tokens, int32_t* cu, int32_t* idx, int64_t idx_len,
+                                     void* workspace, fp2_stream stream) {
+  if (!pl || !seg_count || !blk_idx || !cu || !idx || !workspace) return FP2_ERR_INVALID_ARG;
+  if (tile_tokens != 16 && tile_tokens != 32 && tile_tokens != 64 && tile_tokens != 128) return FP2_ERR_UNSUPPORTED;
+  if (!aligned(workspace, 1024)) return FP2_ERR_INVALID_ARG;
+  if (pl->device < 0) return FP2_ERR_CUDA;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FP2_ERR_CUDA;
+  if (dev != pl->device) return FP2_ERR_INVALID_ARG;
+  const int64_t worst = pl->idx_capacity * (kBlock / tile_tokens);
+  if (worst > 0x7fffffffll) return FP2_ERR_UNSUPPORTED;   // cu is int32
+  if (idx_len < worst) return FP2_ERR_CAPACITY;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  int* status = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(workspace) + pl->ws_status);
+  const int nseg = (int)pl->nseg;
+  pl->last_launches = 0;
+  csr_count_kernel<<<(nseg + 256) / 256, 256, 0, st>>>(pl->d_segs, seg_count, blk_idx, nseg, tile_tokens, cu, status);
+  pl->last_launches += 1;
+  if (nseg > 0) {
+    csr_scan_kernel<<<1, 1024, 0, st>>>(cu, nseg);
+    csr_fill_kernel<<<(unsigned)(((int64_t)nseg * 32 + 255) / 256), 256, 0, st>>>(pl->d_segs, seg_count, blk_idx, nseg,
+                                                                                 tile_tokens, cu, idx, status);
+    pl->last_launches += 2;
+  }
+  return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
+}
+
+extern "C" fp2_status fp2_page_table_from_token_map(fp2_plan* pl, const int32_t* token_to_slot, int32_t max_tokens,
+                                                    const int32_t* seqlens_k, int32_t* page_table, void* workspace,
+                                                    fp2_stream stream) {
+  if (!pl || !token_to_slot || !seqlens_k || !page_table || !workspace || max_tokens <= 0) return FP2_ERR_INVALID_ARG;
+  if (!aligned(workspace, 1024)) return FP2_ERR_INVALID_ARG;
+  if (pl->device < 0) return FP2_ERR_CUDA;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FP2_ERR_CUDA;
+  if (dev != pl->device) return FP2_ERR_INVALID_ARG;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  int* status = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(workspace) + pl->ws_status);
+  const int64_t n = (int64_t)pl->prm.num_seqs * pl->prm.max_pages_per_seq;
+  pl->last_launches = 0;
+  if (n == 0) return FP2_OK;
+  page_table_from_token_map_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(
+      token_to_slot, max_tokens, seqlens_k, pl->prm.num_seqs, pl->prm.page_size, pl->prm.max_pages_per_seq, page_table,
+      status);
+  pl->last_launches = 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
 
