@@ -34,6 +34,12 @@ page-level table taken from a token-level slot map by striding.  Readings: a log
 expands to the physical tiles that hold at least one real token of it (B / tile_tokens of
 them except in a ragged last block); `cu` is the running count in segment order.
 
+KV splitting (Eq. 18; Sec. 3.3 "Sparsity-Aware Load Balancing"): the iteration sequence of a
+segment -- its list backwards (Eq. 17), then its correction terms -- cut into U contiguous
+parts of ceil(n / U) iterations, each part reduced to (O_u, LSE_u) on its own, the parts merged
+by their log-sum-exp weights.  Reading: a correction term belongs to exactly one part (here:
+they follow the listed blocks in the sequence).
+
 Parity pins: every function here is pinned by tests that do not go through this file's
 own formulae (dense limit against a naive loop and torch SDPA, the block-constant closed
 form, brute force on tiny inputs, Eq. 1-3 against Eq. 19-20, invariants).  What is NOT
@@ -416,3 +422,62 @@ def page_table_from_token_map(token_to_slot: np.ndarray, seqlens_k: Sequence[int
             misaligned |= slot % page_size != 0
             pt[b, k] = slot // page_size
     return pt, misaligned
+
+
+# ------------------------------------------------------------------------------------------
+# KV splitting (Eq. 18) and the merge of partial results
+# ------------------------------------------------------------------------------------------
+
+def split_ranges(n: int, U: int):
+    """Eq. 18: part u of U takes iterations [u ceil(n / U), min((u + 1) ceil(n / U), n))."""
+    step = -(-n // U) if n > 0 else 0
+    return [(min(u * step, n), min((u + 1) * step, n)) for u in range(U)]
+
+
+def merge_partials(parts):
+    """parts: [(O_u [rows, d], LSE_u [rows])], LSE_u = -inf (and O_u arbitrary) for an empty part.
+    O = sum_u w_u O_u / sum_u w_u, LSE = log sum_u e^{LSE_u}, w_u = e^{LSE_u - max_u LSE_u}."""
+    lse = np.stack([l for _, l in parts])                       # [U, rows]
+    top = lse.max(axis=0)
+    safe = np.where(np.isfinite(top), top, 0.0)
+    w = np.exp(lse - safe[None, :])                             # e^{-inf} = 0 for empty parts
+    den = w.sum(axis=0)
+    num = sum(w[u][:, None] * np.where(np.isfinite(lse[u])[:, None], parts[u][0], 0.0) for u in range(len(parts)))
+    with np.errstate(divide="ignore", invalid="ignore"):
+        return num / den[:, None], safe + np.log(den)
+
+
+def attend_tile_split(q_tile, pos, K, V, kbar, vbar, n_tok, selected, J_lo, B, scale, use_correction, U):
+    """attend_tile evaluated part by part (Eq. 18) and merged.  The iteration sequence is the listed blocks
+    in descending order (Eq. 17) followed by the corrected blocks in ascending order."""
+    sel = [int(J) for J in selected][::-1]
+    corr = []
+    if use_correction:
+        listed = set(sel)
+        corr = [J for J in range(max(J_lo, 0)) if J not in listed]
+    seq = [("x", J) for J in sel] + [("c", J) for J in corr]
+    Lk = K.shape[0]
+    parts = []
+    for a, b in split_ranges(len(seq), U):
+        logits, values = [], []
+        for kind, J in seq[a:b]:
+            if kind == "x":
+                tok = np.arange(J * B, min((J + 1) * B, Lk))
+                lg = scale * (q_tile @ K[tok].T)
+                logits.append(np.where(tok[None, :] <= pos[:, None], lg, -np.inf))
+                values.append(V[tok])
+            else:
+                logits.append(scale * (q_tile @ kbar[J][:, None]) + math.log(float(n_tok[J])))
+                values.append(vbar[J][None, :])
+        if not logits:
+            parts.append((np.zeros((q_tile.shape[0], V.shape[1])), np.full(q_tile.shape[0], -np.inf)))
+            continue
+        lg = np.concatenate(logits, axis=1)
+        vv = np.concatenate(values, axis=0)
+        m = lg.max(axis=1, keepdims=True)
+        m = np.where(np.isfinite(m), m, 0.0)
+        w = np.exp(lg - m)
+        den = w.sum(axis=1)
+        with np.errstate(divide="ignore", invalid="ignore"):
+            parts.append((np.where(den[:, None] > 0, (w @ vv) / den[:, None], 0.0), m[:, 0] + np.log(den)))
+    return merge_partials(parts)

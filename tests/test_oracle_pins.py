@@ -603,3 +603,49 @@ def test_page_table_from_token_map_round_trip():
     tok[3, 32] += 3                                            # a slot that does not start a page
     got, bad = O.page_table_from_token_map(tok, lens, p, pt.shape[1])
     assert bad
+
+
+# ------------------------------------------------------------------------------------------
+# KV splitting (Eq. 18): the partition is checked against its definition, the merge against
+# the single-pass result and against a two-part case worked by hand
+# ------------------------------------------------------------------------------------------
+
+def test_split_ranges_partition_the_sequence_by_count():
+    for n in range(0, 40):
+        for U in range(1, 9):
+            r = O.split_ranges(n, U)
+            assert len(r) == U
+            covered = [t for a, b in r for t in range(a, b)]
+            assert covered == list(range(n))                    # contiguous, in order, nothing twice
+            sizes = [b - a for a, b in r]
+            assert max(sizes) == -(-n // U)                     # the ceil of Eq. 18
+            assert sizes == sorted(sizes, reverse=True)         # full parts first, then the short one, then empty
+
+
+def test_merge_of_two_parts_by_hand():
+    """Two keys, one per part: weights e^{s0}, e^{s1}; the merge must give the softmax average."""
+    s0, s1 = 0.3, -1.2
+    v0, v1 = np.array([[1.0, 2.0]]), np.array([[-3.0, 0.5]])
+    o, lse = O.merge_partials([(v0, np.array([s0])), (v1, np.array([s1]))])
+    w0, w1 = math.exp(s0), math.exp(s1)
+    assert np.allclose(o, (w0 * v0 + w1 * v1) / (w0 + w1), rtol=0, atol=1e-15)
+    assert abs(lse[0] - math.log(w0 + w1)) < 1e-15
+    o, lse = O.merge_partials([(v0, np.array([s0])), (np.zeros((1, 2)), np.array([-np.inf]))])   # an empty part
+    assert np.allclose(o, v0) and abs(lse[0] - s0) < 1e-15
+
+
+@pytest.mark.parametrize("U", [1, 2, 3, 5, 16])
+@pytest.mark.parametrize("use_correction", [0, 1])
+def test_split_attention_equals_single_pass(U, use_correction):
+    wl, raw = tiny_workload(41, [(700, 200), (130, 0)], Hq=4, Hkv=2, d=16, B=128, M=128, p=16, alpha=0.3,
+                            use_correction=use_correction)
+    sel = O.oracle_select(wl)
+    p = wl.p
+    for s in wl.segs[::3]:
+        K, V, kbar, vbar, n_tok = wl.kv(s.b, s.h)
+        qt = O.tile_queries(wl.q_seq(s.b), p, s)
+        args = (qt, O.row_positions(p, s), K, V, kbar, vbar, n_tok, sel[s.seg][0], s.J_lo, p.block_size, p.scale,
+                use_correction)
+        o1, l1 = O.attend_tile(*args)
+        o2, l2 = O.attend_tile_split(*args, U)
+        assert np.allclose(o1, o2, rtol=0, atol=1e-12) and np.allclose(l1, l2, rtol=0, atol=1e-12)
