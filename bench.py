@@ -307,6 +307,26 @@ def main():
         extra["export_csr"] = {"tile_tokens": 64, "entries": int(2 * sel_pairs), "ms": float(np.mean(exp_ms)),
                                "gbs": exp_bytes / (np.mean(exp_ms) * 1e-3) / 1e9,
                                "note": "3 launches; includes two torch.empty allocations of the helper"}
+        # KV splitting (Eq. 18) on launches with about as many units as workers: attention calls timed with the
+        # split plan on (automatic) and off (the default)
+        if not args.no_sweep:
+            rows = []
+            cases = [("config 1", inputs.config_spec(1)),
+                     ("8192 tokens, Hq=4, Hkv=1", inputs.small_spec(seqs=[(8192, 0)], num_q_heads=4, num_kv_heads=1,
+                                                                    page_size=64, config_id=81)),
+                     ("16384 tokens, Hq=4, Hkv=1", inputs.small_spec(seqs=[(16384, 0)], num_q_heads=4, num_kv_heads=1,
+                                                                     page_size=64, config_id=82))]
+            for name_, sp_ in cases:
+                dcs = binding.DeviceCase(inputs.make_case(sp_))
+                dcs.select()
+                row = {"workload": name_, "segments": dcs.plan.num_segments}
+                for name, tgt in (("auto", 0), ("off", -1)):
+                    dcs.plan.set_split(tgt)
+                    row[f"sparse_us_{name}"] = 1e3 * float(np.median(timed(dcs.sparse, 20, 5)))
+                    row[f"dense_us_{name}"] = 1e3 * float(np.median(timed(dcs.dense, 20, 5)))
+                dcs.status()
+                rows.append(row)
+            extra["split_kv"] = rows
         if not args.no_sweep:
             sweep = []
             for target in (0.5, 0.75, 0.9, 0.95, 0.98):

@@ -151,6 +151,20 @@ fp2_status fp2_dense_prefill_static(fp2_plan* plan, const void* q, const void* k
                                     const int32_t* seqlens_k, const float* q_scale, const float* k_scale,
                                     const float* v_scale, void* out, float* lse, fp2_stream stream);
 
+/* KV splitting (Eq. 18; Sec. 3.3 "Sparsity-Aware Load Balancing"), off by default.  Plans with few segments
+ * (fewer than four per worker CTA of the attention kernel) can cut the iteration sequence of a heavy segment --
+ * its list backwards, then its correction chunks -- into up to 16 contiguous parts of about equal count, run the
+ * parts as separate work units and merge their partial results by log-sum-exp weights; fp2_sparse_prefill and
+ * fp2_dense_prefill then enqueue two more kernels (the device-side split plan and the merge).  The result is the
+ * same up to rounding.
+ *   target < 0 (default): never split;  0: automatic, parts of about the mean load per worker and at least 12
+ *   iterations;  > 0: parts of about `target` iterations (never more than nseg + 2 workers parts in all, which
+ *   is what the workspace is sized for).
+ * Larger plans are never split and ignore the setting; so do calls in which no segment could yield two parts.
+ * On B200 the split did not pay in any case measured (the attention kernel already keeps two independent CTAs per
+ * SM, and the two extra launches cost ~10 us), hence the default.  Host-side, takes effect at the next stage call. */
+fp2_status fp2_plan_set_split(fp2_plan* plan, int32_t target);
+
 /* Index export (Algorithm 1 line 5; Sec. 3.3 "Index-Driven Sparse Traversal", Eq. 17).  Turns the padded lists
  * (seg_count, blk_idx as fp2_select_blocks writes them or as a caller supplies them) into a compact CSR over
  * physical tiles of `tile_tokens` tokens (16, 32, 64 or 128; the paper's kernels use 64): every listed logical

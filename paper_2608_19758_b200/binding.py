@@ -19,7 +19,7 @@ STATUS_NAMES = {0: "FP2_OK", 1: "FP2_ERR_INVALID_ARG", 2: "FP2_ERR_UNSUPPORTED",
 
 EXPORTS = ["fp2_plan_create", "fp2_plan_sizes", "fp2_plan_destroy", "fp2_plan_segment", "fp2_select_blocks",
            "fp2_sparse_prefill", "fp2_dense_prefill", "fp2_dense_prefill_static", "fp2_export_csr",
-           "fp2_page_table_from_token_map", "fp2_read_status", "fp2_last_launch_count", "fp2_status_string"]
+           "fp2_page_table_from_token_map", "fp2_plan_set_split", "fp2_read_status", "fp2_last_launch_count", "fp2_status_string"]
 
 
 class Fp2Error(RuntimeError):
@@ -78,6 +78,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.fp2_export_csr.restype = C.c_int
     lib.fp2_page_table_from_token_map.argtypes = [C.c_void_p, i32p, C.c_int32, i32p, i32p, vp, C.c_void_p]
     lib.fp2_page_table_from_token_map.restype = C.c_int
+    lib.fp2_plan_set_split.argtypes = [C.c_void_p, C.c_int32]
+    lib.fp2_plan_set_split.restype = C.c_int
     lib.fp2_read_status.argtypes = [C.c_void_p, vp, C.POINTER(C.c_int32), C.c_void_p]
     lib.fp2_read_status.restype = C.c_int
     lib.fp2_last_launch_count.argtypes = [C.c_void_p]
@@ -131,6 +133,10 @@ class Plan:
         d = dict(zip(keys, list(out)))
         d["off"] = off.value
         return d
+
+    def set_split(self, target: int):
+        """KV splitting (Eq. 18): < 0 off, 0 automatic, > 0 requested iterations per part."""
+        _check(load().fp2_plan_set_split(self.handle, target), "fp2_plan_set_split")
 
     def last_launch_count(self) -> int:
         return int(load().fp2_last_launch_count(self.handle))

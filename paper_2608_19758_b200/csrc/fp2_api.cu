@@ -36,6 +36,11 @@ struct fp2_plan {
   int32_t* d_blk_off;
   // workspace layout (byte offsets)
   int64_t ws_status, ws_counter, ws_khi, ws_klo, ws_vbar, ws_k8hi, ws_k8lo, ws_order, ws_hist, ws_bytes;
+  // KV splitting (Eq. 18): only plans with few segments carry the buffers
+  bool split_capable;
+  int32_t split_target;   // < 0 off, 0 automatic, > 0 requested iterations per part
+  int32_t max_iters;      // longest iteration sequence any segment can have (all candidates + all chunks)
+  int64_t split_units_cap, ws_unit_seg, ws_unit_split, ws_seg_split, ws_part_ml, ws_part_o;
   EncodeTiledFn encode;
   int32_t last_launches;
   bool attrs_set;
@@ -122,9 +127,12 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
     boff += (lk + kBlock - 1) / kBlock;
   }
   blk_off[p->num_seqs] = (int32_t)boff;
+  pl->max_iters = 0;
   for (int64_t i = 0; i < pl->nseg; ++i) {
     segs[(size_t)i].off = off;
     off += segs[(size_t)i].J_hi + 1;
+    const int iters = segs[(size_t)i].J_hi + 1 + (segs[(size_t)i].J_lo + 127) / 128;
+    pl->max_iters = iters > pl->max_iters ? iters : pl->max_iters;
   }
   pl->idx_capacity = off;
 
@@ -181,6 +189,17 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
   pl->ws_k8lo = o; o += pooled8;
   pl->ws_order = o; o += align_up(4 * (pl->nseg > 0 ? pl->nseg : 1), 1024);
   pl->ws_hist = o;  o += align_up(4 * ((int64_t)p->num_kv_heads * kCountBuckets + 1), 1024);
+  // KV splitting pays when there are fewer units than a few waves of workers; the unit arrays and the partial
+  // results are sized for nseg + 2 workers units, the bound split_plan_kernel keeps
+  const int64_t workers = (int64_t)pl->num_sms * AttnCfg<false>::kCtasPerSm;
+  pl->split_target = -1;   // off unless asked for: see fp2_plan_set_split
+  pl->split_capable = pl->num_sms > 0 && pl->nseg > 0 && pl->nseg < 4 * workers && pl->nseg + 2 * workers < 65536;
+  pl->split_units_cap = pl->split_capable ? pl->nseg + 2 * workers : 0;
+  pl->ws_unit_seg = o;   o += align_up(4 * pl->split_units_cap, 1024);
+  pl->ws_unit_split = o; o += align_up(4 * pl->split_units_cap, 1024);
+  pl->ws_seg_split = o;  o += align_up(pl->split_capable ? 8 * pl->nseg : 0, 1024);   // per-segment word + list of split segments
+  pl->ws_part_ml = o;    o += align_up(pl->split_units_cap * 128 * 8, 1024);
+  pl->ws_part_o = o;     o += pl->split_units_cap * 128 * 128 * 4;
   pl->ws_bytes = o;
 
   DevParams& d = pl->dev;
@@ -219,6 +238,12 @@ extern "C" fp2_status fp2_plan_segment(const fp2_plan* pl, int64_t seg, int32_t*
   const int32_t v[10] = {s.b, s.h, s.t, s.r0, s.nrows, s.pre, s.Lk, s.J_lo, s.J_hi, s.blk_off};
   memcpy(out10, v, sizeof(v));
   if (list_offset) *list_offset = s.off;
+  return FP2_OK;
+}
+
+extern "C" fp2_status fp2_plan_set_split(fp2_plan* pl, int32_t target) {
+  if (!pl) return FP2_ERR_INVALID_ARG;
+  pl->split_target = target;
   return FP2_OK;
 }
 
@@ -348,9 +373,10 @@ extern "C" fp2_status fp2_select_blocks(fp2_plan* pl, const void* q, const void*
 // Attention: two 256-thread CTAs per SM, each a persistent worker on the shared work counter.  mkb / mkb_lo:
 // pooled keys of the correction chunks (BF16: one BF16 array, mkb_lo unused; FP8: e4m3 hi and lo).
 static void launch_attn(fp2_plan* pl, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mkb,
-                        const CUtensorMap& mkb_lo, const CUtensorMap& mvb, const AttnArgs& a, cudaStream_t st) {
+                        const CUtensorMap& mkb_lo, const CUtensorMap& mvb, const AttnArgs& a, int64_t max_units,
+                        cudaStream_t st) {
   const int64_t workers = (int64_t)pl->num_sms * AttnCfg<false>::kCtasPerSm;
-  const unsigned grid = (unsigned)(pl->nseg < workers ? pl->nseg : workers);
+  const unsigned grid = (unsigned)(max_units < workers ? max_units : workers);
   if (pl->dev.fp8)
     sparse_attn_kernel<true><<<grid, AttnCfg<true>::kThreads, AttnCfg<true>::kSmemBytes, st>>>(mk, mv, mkb, mkb_lo,
                                                                                                  mvb, a, pl->dev);
@@ -399,8 +425,41 @@ static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, cons
   a.lse = lse;
   a.work_counter = reinterpret_cast<int*>(ws + pl->ws_counter);
   a.status = reinterpret_cast<int*>(ws + pl->ws_status);
-  launch_attn(pl, mk, mv, mkb, mkb_lo, mvb, a, st);
+  a.unit_split = nullptr; a.n_units = nullptr; a.part_o = nullptr; a.part_ml = nullptr;
+  // a part is never shorter than kMinPartLen iterations (or the requested length): nothing to split when even the
+  // longest candidate range (plus its correction chunks) is below one and a half such parts
+  const int min_len = pl->split_target > 0 ? pl->split_target : kMinPartLen;
+  const bool split = pl->split_capable && pl->split_target >= 0 && 2 * pl->max_iters >= 3 * min_len;
+  int64_t max_units = pl->nseg;
+  if (split) {
+    // device-side scheduler prep (Eq. 18): units = parts of segments, in the work order
+    int32_t* unit_seg = reinterpret_cast<int32_t*>(ws + pl->ws_unit_seg);
+    int32_t* unit_split = reinterpret_cast<int32_t*>(ws + pl->ws_unit_split);
+    int32_t* seg_split = reinterpret_cast<int32_t*>(ws + pl->ws_seg_split);
+    int32_t* split_list = seg_split + pl->nseg;
+    int32_t* n_units = reinterpret_cast<int32_t*>(ws + pl->ws_counter) + 1;
+    int32_t* n_split = n_units + 1;
+    const int workers = pl->num_sms * AttnCfg<false>::kCtasPerSm;
+    split_plan_kernel<<<1, 1024, 0, st>>>(pl->d_segs, a.order, seg_count, (int)pl->nseg, pl->dev.use_correction,
+                                          workers, pl->split_target, unit_seg, unit_split, seg_split, split_list, n_units,
+                                          n_split);
+    pl->last_launches += 1;
+    a.order = unit_seg;
+    a.unit_split = unit_split;
+    a.n_units = n_units;
+    a.part_o = reinterpret_cast<float*>(ws + pl->ws_part_o);
+    a.part_ml = reinterpret_cast<float2*>(ws + pl->ws_part_ml);
+    max_units = pl->split_units_cap;
+  }
+  launch_attn(pl, mk, mv, mkb, mkb_lo, mvb, a, max_units, st);
   pl->last_launches += 1;
+  if (split) {
+    int32_t* seg_split = reinterpret_cast<int32_t*>(ws + pl->ws_seg_split);
+    split_combine_kernel<<<(unsigned)(pl->num_sms * 8), 128, 0, st>>>(
+        pl->d_segs, seg_split, seg_split + pl->nseg, reinterpret_cast<int32_t*>(ws + pl->ws_counter) + 2, a.part_o,
+        a.part_ml, fp8 ? vs : nullptr, pl->dev, a.out, lse);
+    pl->last_launches += 1;
+  }
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
 
@@ -497,7 +556,8 @@ extern "C" fp2_status fp2_dense_prefill_static(fp2_plan* pl, const void* q, cons
   a.work_counter = reinterpret_cast<int*>(sw + 64);
   a.status = reinterpret_cast<int*>(sw);
   // the dense path stages no pooled chunks: the two pooled-mean maps are never dereferenced
-  launch_attn(pl, mk, mv, mk, mk, mv, a, st);
+  a.unit_split = nullptr; a.n_units = nullptr; a.part_o = nullptr; a.part_ml = nullptr;
+  launch_attn(pl, mk, mv, mk, mk, mv, a, pl->nseg, st);
   pl->last_launches = 4;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }

@@ -42,6 +42,7 @@
 #include "common.cuh"
 #include "ptx.cuh"
 #include "score_select.cuh"  // load_q_tile_async
+#include "split_kv.cuh"
 
 namespace fp2 {
 
@@ -54,6 +55,9 @@ struct TileInfo {
   int32_t T;         // exact iterations (listed blocks)
   int32_t nchunk;    // non-empty correction chunks
   int32_t dense;
+  int32_t it_begin, it_end;   // this unit's part of the iteration sequence [0, T + nchunk) (Eq. 18); all of it unless split
+  int32_t parts;              // parts the segment is split into (1: the unit writes the final output)
+  int32_t slot;               // partial-result slot of this unit when parts > 1
   int32_t chunk_id[kMaxChunks];
   uint32_t todo[kMaxChunks][4];
 };
@@ -72,6 +76,13 @@ struct AttnArgs {
   float* lse;
   int* work_counter;
   int* status;
+  // KV splitting (Eq. 18).  unit_split == NULL: one unit per segment, `order` lists the segments.  Otherwise
+  // `order` lists the segment of every unit, unit_split its part (see pack_split), *n_units their number, and a
+  // unit of a split segment leaves (O, m, l) unnormalised in part_o [slot][128][128] / part_ml [slot][128].
+  const int32_t* unit_split;
+  const int32_t* n_units;
+  float* part_o;
+  float2* part_ml;
 };
 
 constexpr int kPParts = 4;   // P is handed to the issuer in this many column slices (4 or 8)
@@ -248,8 +259,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       TileInfo& ti = info[slot];
       if (t64 == 0) {
         const int w = atomicAdd(A.work_counter, 1);
-        if (w < P.nseg) {
+        const int n_units = A.unit_split ? *A.n_units : P.nseg;
+        if (w < n_units) {
           const int seg = A.order[w];
+          const int32_t split = A.unit_split ? A.unit_split[w] : pack_split(0, 1, 0);
+          ti.parts = (split >> 8) & 0xff;
+          ti.slot = ((split >> 16) & 0xffff) + (split & 0xff);
+          ti.it_begin = split & 0xff;   // the part index for now; turned into a range once T + nchunk is known
           ti.sg = A.segs[seg];
           ti.valid = 1;
           ti.dense = (A.seg_count == nullptr);
@@ -305,6 +321,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         }
       }
       named_bar_sync(2, kSetupThreads);
+      if (t64 == 0 && valid) {   // Eq. 18: part u of U takes iterations [u ceil(n / U), min((u + 1) ceil(n / U), n))
+        const int n = ti.T + ti.nchunk, u = ti.it_begin;
+        const int step = (n + ti.parts - 1) / ti.parts;
+        ti.it_begin = min(u * step, n);
+        ti.it_end = min((u + 1) * step, n);
+      }
+      named_bar_sync(2, kSetupThreads);
       if (t64 == 0) mbar_arrive(&info_full[slot]);
       if (!valid) break;
       // Q tile: wait until every S = Q K^T of the previous unit has completed, then overwrite
@@ -336,7 +359,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       const TileInfo& ti = info[slot];
       if (!ti.valid) break;
       const SegInfo& sg = ti.sg;
-      const int T = ti.T, n_it = T + ti.nchunk;
+      const int T = ti.T;
       const int32_t* list = A.blk_idx + sg.off;
       const int32_t* pt = A.page_table + (size_t)sg.b * P.max_pages_per_seq;
       // page id of this lane's page of exact iteration i (-1: past the end of the sequence, or not an exact
@@ -353,8 +376,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         }
         return pid;
       };
-      int pid_next = fetch_pid(0);
-      for (int i = 0; i < n_it; ++i, ++G) {
+      int pid_next = fetch_pid(ti.it_begin);
+      for (int i = ti.it_begin; i < ti.it_end; ++i, ++G) {
         const int pid = pid_next;
         pid_next = fetch_pid(i + 1);
         if (G >= 1) mbar_wait(&s_done, (G - 1) & 1, ctx, 302);   // K stage free
@@ -426,10 +449,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 403);
         const TileInfo& ti = info[slot];
         if (!ti.valid) break;
-        const int T = ti.T, n_it = T + ti.nchunk;
+        const int T = ti.T;
         (void)T;
         mbar_wait(&q_full, it & 1, ctx, 404);
-        for (int i = 0; i < n_it; ++i, ++G) {
+        const int i0 = ti.it_begin, i1 = ti.it_end;
+        for (int i = i0; i < i1; ++i, ++G) {
           // S = Q K^T (G).  The S columns are free: O += P V (G-1), which read P out of them, was issued before.
           mbar_wait(&k_full, G & 1, ctx, 405);
           tc_fence_after();
@@ -455,7 +479,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
             }
           }
           umma_commit(&s_done);
-          if (i == n_it - 1) umma_commit(&q_empty);
+          if (i == i1 - 1) umma_commit(&q_empty);
           // O += P V (G)
           mbar_wait(&v_full, G & 1, ctx, 402);
 #pragma unroll
@@ -465,12 +489,12 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
 #pragma unroll
             for (int ks = (8 / kPParts) * h; ks < (8 / kPParts) * (h + 1); ++ks) {
               const uint64_t bd = make_smem_desc_sw128(v_addr + ks * 2048, 16384, 1024);
-              umma_f16_ts(tmem + 128, tmem + ks * 8, bd, idesc_pv, (i > 0) || ks > 0);
+              umma_f16_ts(tmem + 128, tmem + ks * 8, bd, idesc_pv, (i > i0) || ks > 0);
             }
           }
           umma_commit(&pv_done[G & 1]);
         }
-        if (n_it == 0) umma_commit(&q_empty);  // empty list: nothing read Q, release it at once
+        if (i1 == i0) umma_commit(&q_empty);  // nothing to do for this unit: nothing read Q, release it at once
         mbar_arrive(&info_empty[slot]);
       }
     }
@@ -489,7 +513,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 501);
       const TileInfo& ti = info[slot];
       if (!ti.valid) break;
-      const int T = ti.T, n_it = T + ti.nchunk;
+      const int T = ti.T;
       const bool dense = ti.dense != 0;
       const int J_hi = ti.sg.J_hi, J_lo = ti.sg.J_lo;
       const int32_t* list = A.blk_idx + ti.sg.off;
@@ -504,8 +528,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       }
       float m = -INFINITY, l = 0.f;
       // block id of the next exact iteration, fetched one iteration ahead
-      int J_next = (!dense && T > 0) ? list[T - 1] : 0;
-      for (int i = 0; i < n_it; ++i, ++G) {
+      const int i0 = ti.it_begin, i1 = ti.it_end;
+      int J_next = (!dense && i0 < T) ? list[T - 1 - i0] : 0;
+      for (int i = i0; i < i1; ++i, ++G) {
         // iteration kind and masks
         bool need_mask = false;
         int tok_lim = 1 << 30;     // exact block: columns j with j <= tok_lim are visible
@@ -554,7 +579,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         // MMAs complete in issue order, so S (G) in TMEM means O += P V (G-1) has been added.
         if (__any_sync(0xffffffffu, m_new > m + 8.0f)) {
           const float f = (m == -INFINITY) ? 0.f : ex2(m - m_new);
-          if (i > 0) {
+          if (i > i0) {
 #pragma unroll 1
             for (int k = 0; k < 4; ++k) {
               uint32_t rr[32];
@@ -578,7 +603,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       // ------------------------------ epilogue ------------------------------
       const SegInfo& sg = ti.sg;
       const float inv = l > 0.f ? out_scale / l : 0.f;
-      const bool have_o = n_it >= 1;
+      const bool have_o = i1 > i0;
       const bool row_ok = row < sg.nrows;
       const size_t tok = (size_t)sg.q_tok0 + r / g;
       const int head = sg.h * g + r % g;
@@ -586,6 +611,24 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       if (have_o) {
         wait_pv(G - 1, 503);   // O += P V of the unit's last iteration
         tc_fence_after();
+      }
+      if (ti.parts > 1) {
+        // one part of a split segment (Eq. 18): leave (O, m, l) unnormalised for the merge kernel
+        float* prow = A.part_o + ((size_t)ti.slot * 128 + row) * 128;
+        if (have_o) {
+#pragma unroll 1
+          for (int k = 0; k < 4; ++k) {
+            uint32_t a0[32];
+            tmem_ld32(o_addr + k * 32, a0);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 4; ++j) st_global_v8(prow + k * 32 + j * 8, &a0[j * 8], stream_pol);
+          }
+        }
+        A.part_ml[(size_t)ti.slot * 128 + row] = make_float2(have_o ? m : -INFINITY, have_o ? l : 0.f);
+        tc_fence_before();
+        mbar_arrive(&info_empty[slot]);
+        continue;
       }
 #pragma unroll 1
       for (int k = 0; k < 4; ++k) {

@@ -350,3 +350,6 @@ def test_launch_counts_are_reported():
     assert dc.plan.last_launch_count() == 2           # pool + score/select
     dc.sparse()
     assert dc.plan.last_launch_count() == 4           # order (3) + attention
+    dc.plan.set_split(4)
+    dc.sparse()
+    assert dc.plan.last_launch_count() == 6           # order (3) + split plan + attention + merge
