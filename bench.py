@@ -327,6 +327,28 @@ def main():
                 dcs.status()
                 rows.append(row)
             extra["split_kv"] = rows
+        # chunked prefill (Sec. 4.3): the last 8K-token chunk of a 128K-token sequence; the index stage with the
+        # prefix pooled again against the prefix's pooled means carried over from the previous chunk
+        if not args.no_sweep and args.config == 3 and args.scale_down == 1:
+            import copy
+            sp_prev = copy.deepcopy(spec); sp_prev.seqs = [(122880, 114688)]
+            sp_last = copy.deepcopy(spec); sp_last.seqs = [(131072, 122880)]
+            c_last = inputs.make_case(sp_last)
+            c_prev = copy.copy(c_last)     # same KV pool and page table; queries of the previous chunk do not matter here
+            c_prev.spec = sp_prev
+            c_prev.seqlens_k = torch.tensor([122880], dtype=torch.int32)
+            d_prev, d_last = binding.DeviceCase(c_prev), binding.DeviceCase(c_last)
+            d_prev.select()
+
+            def carried():
+                binding.fp2_pool_carry(d_last.plan, d_last.workspace, d_prev.plan, d_prev.workspace, [0])
+                d_last.select()
+            t_fresh = float(np.median(timed(d_last.select, 10, 3)))
+            t_carry = float(np.median(timed(carried, 10, 3)))
+            d_last.status()
+            extra["chunked_prefill"] = {"workload": "last 8192-token chunk of 131072 tokens, Hq=32 Hkv=8",
+                                        "select_ms_pool_all": t_fresh, "select_ms_with_carry": t_carry,
+                                        "blocks_carried": 960, "blocks_pooled": 64}
         if not args.no_sweep:
             sweep = []
             for target in (0.5, 0.75, 0.9, 0.95, 0.98):

@@ -151,6 +151,22 @@ fp2_status fp2_dense_prefill_static(fp2_plan* plan, const void* q, const void* k
                                     const int32_t* seqlens_k, const float* q_scale, const float* k_scale,
                                     const float* v_scale, void* out, float* lse, fp2_stream stream);
 
+/* Pooled statistics carried over between the chunks of a chunked prefill (Sec. 4.3 "Compatibility with Chunked
+ * Prefill": the index stage is re-run for every chunk; pooling the cached prefix again each time is avoidable work).  `src` /
+ * `src_workspace` are the plan and workspace of the previous chunk after its fp2_select_blocks; `dst` is this
+ * chunk's plan.  h_src_seq (HOST, dst.num_seqs entries) names for every sequence of `dst` its index in `src`, or
+ * -1 for a sequence that was not there.  For every block that was complete then and is complete now
+ * (floor(min(Lk_src, Lk_dst) / 128) per sequence) the pooled means are copied from src_workspace to
+ * dst_workspace, and the next fp2_select_blocks on `dst` -- only that one -- pools just the remaining blocks.
+ * The caller guarantees that those blocks hold the same K / V (and, for FP8, the same scales) as before, which is
+ * what a paged prefix cache does.  Plans must agree in KV heads and dtype.  One copy kernel on `stream`; the
+ * stream must be ordered after the previous chunk's fp2_select_blocks and before dst's.  Nothing is allocated.
+ * fp2_pool_carry_count is the host-side half alone: h_blocks[b] = blocks that would be carried (needs no device). */
+fp2_status fp2_pool_carry(fp2_plan* dst, void* dst_workspace, const fp2_plan* src, const void* src_workspace,
+                          const int32_t* h_src_seq, fp2_stream stream);
+fp2_status fp2_pool_carry_count(const fp2_plan* dst, const fp2_plan* src, const int32_t* h_src_seq,
+                                int32_t* h_blocks);
+
 /* KV splitting (Eq. 18; Sec. 3.3 "Sparsity-Aware Load Balancing"), off by default.  Plans with few segments
  * (fewer than four per worker CTA of the attention kernel) can cut the iteration sequence of a heavy segment --
  * its list backwards, then its correction chunks -- into up to 16 contiguous parts of about equal count, run the
@@ -178,7 +194,7 @@ fp2_status fp2_plan_set_split(fp2_plan* plan, int32_t target);
 fp2_status fp2_export_csr(fp2_plan* plan, const int32_t* seg_count, const int32_t* blk_idx, int32_t tile_tokens,
                           int32_t* cu, int32_t* idx, int64_t idx_len, void* workspace, fp2_stream stream);
 
-/* Page-level table from a token-level slot map (Sec. 4.4 "Serving Integration": the page index is the token-level
+/* Page-level table from a token-level slot map (Sec. 3.4 "Serving Integration": the page index is the token-level
  * mapping read every page_size entries; Eq. 22 is the inverse).  token_to_slot int32 [num_seqs, max_tokens] holds
  * the global slot (page * page_size + offset) of token j of sequence b; entries past seqlens_k[b] are not read.
  *   out: page_table int32 [num_seqs, max_pages_per_seq], -1 for pages past the end of a sequence.

@@ -28,7 +28,7 @@ forms):
   * comparison is ">=": equality selects;
   * LSE is the natural log of the corrected denominator, softmax scale included.
 
-Index export (Algorithm 1 line 5; Sec. 3.3 "Index-Driven Sparse Traversal", Eq. 17; Sec. 4.4
+Index export (Algorithm 1 line 5; Sec. 3.3 "Index-Driven Sparse Traversal", Eq. 17; Sec. 3.4
 "Serving Integration"): the block lists as a compact CSR of physical tiles, and the
 page-level table taken from a token-level slot map by striding.  Readings: a logical block
 expands to the physical tiles that hold at least one real token of it (B / tile_tokens of
@@ -407,7 +407,7 @@ def export_csr(wl: Workload, lists, tile_tokens: int = 64):
 
 def page_table_from_token_map(token_to_slot: np.ndarray, seqlens_k: Sequence[int], page_size: int,
                               max_pages: int):
-    """Sec. 4.4: the page-level table is the token-level slot map read every page_size entries.
+    """Sec. 3.4: the page-level table is the token-level slot map read every page_size entries.
     token_to_slot [ns, max_tokens]: global slot of token j of sequence b (Eq. 22's addr(b, j)).
     Returns (page_table int32 [ns, max_pages] with -1 past the last page, misaligned) where misaligned
     says some sampled slot was not the first slot of a page."""

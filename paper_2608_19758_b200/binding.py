@@ -19,7 +19,8 @@ STATUS_NAMES = {0: "FP2_OK", 1: "FP2_ERR_INVALID_ARG", 2: "FP2_ERR_UNSUPPORTED",
 
 EXPORTS = ["fp2_plan_create", "fp2_plan_sizes", "fp2_plan_destroy", "fp2_plan_segment", "fp2_select_blocks",
            "fp2_sparse_prefill", "fp2_dense_prefill", "fp2_dense_prefill_static", "fp2_export_csr",
-           "fp2_page_table_from_token_map", "fp2_plan_set_split", "fp2_read_status", "fp2_last_launch_count", "fp2_status_string"]
+           "fp2_page_table_from_token_map", "fp2_plan_set_split", "fp2_pool_carry", "fp2_pool_carry_count",
+           "fp2_read_status", "fp2_last_launch_count", "fp2_status_string"]
 
 
 class Fp2Error(RuntimeError):
@@ -78,6 +79,10 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.fp2_export_csr.restype = C.c_int
     lib.fp2_page_table_from_token_map.argtypes = [C.c_void_p, i32p, C.c_int32, i32p, i32p, vp, C.c_void_p]
     lib.fp2_page_table_from_token_map.restype = C.c_int
+    lib.fp2_pool_carry.argtypes = [C.c_void_p, vp, C.c_void_p, vp, C.POINTER(C.c_int32), C.c_void_p]
+    lib.fp2_pool_carry.restype = C.c_int
+    lib.fp2_pool_carry_count.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.fp2_pool_carry_count.restype = C.c_int
     lib.fp2_plan_set_split.argtypes = [C.c_void_p, C.c_int32]
     lib.fp2_plan_set_split.restype = C.c_int
     lib.fp2_read_status.argtypes = [C.c_void_p, vp, C.POINTER(C.c_int32), C.c_void_p]
@@ -214,6 +219,23 @@ def fp2_page_table_from_token_map(plan: Plan, token_to_slot, seqlens_k, page_tab
     _check(load().fp2_page_table_from_token_map(plan.handle, _ptr(token_to_slot), token_to_slot.shape[1],
                                                 _ptr(seqlens_k), _ptr(page_table), _ptr(workspace),
                                                 _stream(stream)), "fp2_page_table_from_token_map")
+
+
+def fp2_pool_carry_count(dst: Plan, src: Plan, src_seq):
+    """Blocks per sequence of `dst` whose pooled means would be carried over from `src` (host only)."""
+    ns = len(src_seq)
+    a = (C.c_int32 * max(ns, 1))(*src_seq)
+    out = (C.c_int32 * max(ns, 1))()
+    _check(load().fp2_pool_carry_count(dst.handle, src.handle, a, out), "fp2_pool_carry_count")
+    return list(out)[:ns]
+
+
+def fp2_pool_carry(dst: Plan, dst_workspace, src: Plan, src_workspace, src_seq, stream=None):
+    """Copies the pooled means of the blocks complete in both chunks from src_workspace to dst_workspace; the next
+    fp2_select_blocks on `dst` pools only the rest."""
+    a = (C.c_int32 * max(len(src_seq), 1))(*src_seq)
+    _check(load().fp2_pool_carry(dst.handle, _ptr(dst_workspace), src.handle, _ptr(src_workspace), a,
+                                 _stream(stream)), "fp2_pool_carry")
 
 
 def fp2_read_status(plan: Plan, workspace, stream=None, raise_on_error: bool = True):

@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include <new>
+#include <algorithm>
 #include <vector>
 
 #include "../../include/fp2.h"
@@ -34,6 +35,9 @@ struct fp2_plan {
   void* d_table;
   SegInfo* d_segs;
   int32_t* d_blk_off;
+  int32_t* d_carry;                 // [3 x num_seqs]: pooled rows carried over from a previous chunk (fp2_pool_carry)
+  std::vector<int32_t> h_blk_off, h_carry;
+  bool carry_valid;
   // workspace layout (byte offsets)
   int64_t ws_status, ws_counter, ws_khi, ws_klo, ws_vbar, ws_k8hi, ws_k8lo, ws_order, ws_hist, ws_bytes;
   // KV splitting (Eq. 18): only plans with few segments carry the buffers
@@ -135,6 +139,9 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
     pl->max_iters = iters > pl->max_iters ? iters : pl->max_iters;
   }
   pl->idx_capacity = off;
+  pl->h_blk_off = blk_off;
+  pl->carry_valid = false;
+  pl->d_carry = nullptr;
 
   // Device part.  Without a usable CUDA device the plan is still returned (sizes and the segment table can be
   // queried), but every stage call on it fails with FP2_ERR_CUDA.
@@ -148,10 +155,12 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
     pl->device = dev;
     pl->num_sms = prop.multiProcessorCount;
     const size_t seg_bytes = (size_t)align_up((int64_t)sizeof(SegInfo) * (pl->nseg > 0 ? pl->nseg : 1), 256);
-    const size_t tab_bytes = seg_bytes + sizeof(int32_t) * blk_off.size();
+    const size_t boff_bytes = (size_t)align_up((int64_t)sizeof(int32_t) * blk_off.size(), 256);
+    const size_t tab_bytes = seg_bytes + boff_bytes + sizeof(int32_t) * 3 * (p->num_seqs > 0 ? p->num_seqs : 1);
     if (cudaMalloc(&pl->d_table, tab_bytes) != cudaSuccess) { delete pl; return FP2_ERR_CUDA; }
     pl->d_segs = reinterpret_cast<SegInfo*>(pl->d_table);
     pl->d_blk_off = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(pl->d_table) + seg_bytes);
+    pl->d_carry = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(pl->d_table) + seg_bytes + boff_bytes);
     if ((pl->nseg > 0 && cudaMemcpy(pl->d_segs, segs.data(), sizeof(SegInfo) * segs.size(),
                                     cudaMemcpyHostToDevice) != cudaSuccess) ||
         cudaMemcpy(pl->d_blk_off, blk_off.data(), sizeof(int32_t) * blk_off.size(), cudaMemcpyHostToDevice) !=
@@ -304,7 +313,8 @@ static fp2_status check_common(fp2_plan* pl, const void* q, const void* k, const
 }
 
 static fp2_status launch_pool(fp2_plan* pl, const void* k, const void* v, const int32_t* pt, const int32_t* lk,
-                              const float* ks, const float* vs, uint8_t* ws, cudaStream_t st) {
+                              const float* ks, const float* vs, uint8_t* ws, cudaStream_t st,
+                              const int32_t* carry = nullptr) {
   if (pl->nblk_tot == 0) return FP2_OK;
   const unsigned grid = (unsigned)(pl->nblk_tot * pl->prm.num_kv_heads * 2);   // K and V pooled by separate CTAs
   __nv_bfloat16* khi = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_khi);
@@ -312,10 +322,10 @@ static fp2_status launch_pool(fp2_plan* pl, const void* k, const void* v, const 
   __nv_bfloat16* vb = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_vbar);
   if (pl->dev.fp8)
     pool_kv_kernel<true><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, lk, pl->d_blk_off, ks, vs,
-                                               pl->dev, khi, klo, vb, ws + pl->ws_k8hi, ws + pl->ws_k8lo);
+                                               pl->dev, khi, klo, vb, ws + pl->ws_k8hi, ws + pl->ws_k8lo, carry);
   else
     pool_kv_kernel<false><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, lk, pl->d_blk_off, ks, vs,
-                                                pl->dev, khi, klo, vb, nullptr, nullptr);
+                                                pl->dev, khi, klo, vb, nullptr, nullptr, carry);
   pl->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
@@ -350,7 +360,10 @@ extern "C" fp2_status fp2_select_blocks(fp2_plan* pl, const void* q, const void*
   uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
   pl->last_launches = 0;
   if (pl->nseg == 0) return FP2_OK;
-  if ((s = launch_pool(pl, k, v, pt, lk, ks, vs, ws, st)) != FP2_OK) return s;
+  // pooled rows carried over by fp2_pool_carry are used once: by this call
+  const int32_t* carry = pl->carry_valid ? pl->d_carry : nullptr;
+  pl->carry_valid = false;
+  if ((s = launch_pool(pl, k, v, pt, lk, ks, vs, ws, st, carry)) != FP2_OK) return s;
   CUtensorMap mhi, mlo;
   if (!make_map(pl, &mhi, ws + pl->ws_khi, pl->nblk_tot, pl->prm.num_kv_heads, 128, false) ||
       !make_map(pl, &mlo, ws + pl->ws_klo, pl->nblk_tot, pl->prm.num_kv_heads, 128, false))
@@ -559,6 +572,63 @@ extern "C" fp2_status fp2_dense_prefill_static(fp2_plan* pl, const void* q, cons
   a.unit_split = nullptr; a.n_units = nullptr; a.part_o = nullptr; a.part_ml = nullptr;
   launch_attn(pl, mk, mv, mk, mk, mv, a, pl->nseg, st);
   pl->last_launches = 4;
+  return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Pooled statistics carried from the previous chunk of a chunked prefill
+// ------------------------------------------------------------------------------------------------------
+extern "C" fp2_status fp2_pool_carry_count(const fp2_plan* dst, const fp2_plan* src, const int32_t* h_src_seq,
+                                           int32_t* h_blocks) {
+  if (!dst || !src || !h_src_seq || !h_blocks) return FP2_ERR_INVALID_ARG;
+  if (dst->prm.num_kv_heads != src->prm.num_kv_heads || dst->prm.dtype != src->prm.dtype) return FP2_ERR_INVALID_ARG;
+  for (int b = 0; b < dst->prm.num_seqs; ++b) {
+    const int s = h_src_seq[b];
+    if (s >= src->prm.num_seqs) return FP2_ERR_INVALID_ARG;
+    // a block's means carry over if the block was complete then and is complete now
+    h_blocks[b] = s < 0 ? 0 : std::min(src->h_lk[(size_t)s], dst->h_lk[(size_t)b]) / kBlock;
+  }
+  return FP2_OK;
+}
+
+extern "C" fp2_status fp2_pool_carry(fp2_plan* dst, void* dst_workspace, const fp2_plan* src,
+                                     const void* src_workspace, const int32_t* h_src_seq, fp2_stream stream) {
+  if (!dst || !src || !dst_workspace || !src_workspace || !h_src_seq) return FP2_ERR_INVALID_ARG;
+  if (!aligned(dst_workspace, 1024) || !aligned(src_workspace, 1024)) return FP2_ERR_INVALID_ARG;
+  if (dst->device < 0 || src->device != dst->device) return FP2_ERR_CUDA;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FP2_ERR_CUDA;
+  if (dev != dst->device) return FP2_ERR_INVALID_ARG;
+  const int ns = dst->prm.num_seqs;
+  dst->h_carry.assign((size_t)3 * (ns > 0 ? ns : 1), 0);
+  std::vector<int32_t> n((size_t)(ns > 0 ? ns : 1));
+  fp2_status s = fp2_pool_carry_count(dst, src, h_src_seq, n.data());
+  if (s != FP2_OK) return s;
+  int max_n = 0;
+  for (int b = 0; b < ns; ++b) {
+    dst->h_carry[3 * b] = h_src_seq[b] < 0 ? 0 : src->h_blk_off[(size_t)h_src_seq[b]];
+    dst->h_carry[3 * b + 1] = dst->h_blk_off[(size_t)b];
+    dst->h_carry[3 * b + 2] = n[(size_t)b];
+    max_n = std::max(max_n, n[(size_t)b]);
+  }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  dst->last_launches = 0;
+  if (ns == 0) return FP2_OK;
+  // (a pageable host source: the runtime stages the bytes before this call returns)
+  if (cudaMemcpyAsync(dst->d_carry, dst->h_carry.data(), sizeof(int32_t) * 3 * ns, cudaMemcpyHostToDevice, st) !=
+      cudaSuccess)
+    return FP2_ERR_CUDA;
+  dst->carry_valid = true;
+  if (max_n == 0) return FP2_OK;
+  const uint8_t* sw = reinterpret_cast<const uint8_t*>(src_workspace);
+  uint8_t* dw = reinterpret_cast<uint8_t*>(dst_workspace);
+  const int rb16 = dst->prm.num_kv_heads * kHeadDim * 2;
+  const int rb8 = dst->dev.fp8 ? dst->prm.num_kv_heads * kHeadDim : 0;
+  const unsigned gy = (unsigned)std::min((max_n + 7) / 8, 1024);
+  pool_carry_kernel<<<dim3((unsigned)ns, gy), 256, 0, st>>>(
+      dst->d_carry, rb16, rb8, sw + src->ws_khi, sw + src->ws_klo, sw + src->ws_vbar, sw + src->ws_k8hi,
+      sw + src->ws_k8lo, dw + dst->ws_khi, dw + dst->ws_klo, dw + dst->ws_vbar, dw + dst->ws_k8hi, dw + dst->ws_k8lo);
+  dst->last_launches = 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
 

@@ -1,4 +1,4 @@
-// Index export (Algorithm 1 line 5; Sec. 3.3 "Index-Driven Sparse Traversal", Eq. 17; Sec. 4.4 "Serving
+// Index export (Algorithm 1 line 5; Sec. 3.3 "Index-Driven Sparse Traversal", Eq. 17; Sec. 3.4 "Serving
 // Integration"): the padded block lists of the selector as a compact CSR (cu, idx) of physical tiles of
 // tile_tokens tokens, per segment in segment order (that is: per KV head under PackGQA), and the page-level
 // table read out of a token-level slot map by striding.
@@ -93,7 +93,7 @@ __global__ void csr_fill_kernel(const SegInfo* __restrict__ segs, const int32_t*
   if (bad) atomicOr(status + ST_BAD_LIST, 1);
 }
 
-// page_table[b][k] = token_to_slot[b][k p] / p for the pages that hold a token, -1 beyond (Sec. 4.4).  A sampled
+// page_table[b][k] = token_to_slot[b][k p] / p for the pages that hold a token, -1 beyond (Sec. 3.4).  A sampled
 // slot that is not the first of a page is flagged in the status block.
 __global__ void page_table_from_token_map_kernel(const int32_t* __restrict__ token_to_slot, int max_tokens,
                                                  const int32_t* __restrict__ seqlens_k, int ns, int p, int max_pages,

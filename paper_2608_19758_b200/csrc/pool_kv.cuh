@@ -57,7 +57,8 @@ __global__ void __launch_bounds__(256, 4) pool_kv_kernel(const uint8_t* __restri
                                                          __nv_bfloat16* __restrict__ kbar_lo,
                                                          __nv_bfloat16* __restrict__ vbar,
                                                          uint8_t* __restrict__ kbar8_hi,
-                                                         uint8_t* __restrict__ kbar8_lo) {
+                                                         uint8_t* __restrict__ kbar8_lo,
+                                                         const int32_t* __restrict__ carry) {
   constexpr int ROW_BYTES = FP8 ? 128 : 256;
   constexpr int CHUNKS = ROW_BYTES / 16;       // 16-byte chunks per token row
   constexpr int EPC = FP8 ? 16 : 8;            // elements per chunk
@@ -76,6 +77,9 @@ __global__ void __launch_bounds__(256, 4) pool_kv_kernel(const uint8_t* __restri
     if (blk_off[mid] <= gblk) lo = mid; else hi = mid;
   }
   const int b = lo, J = gblk - blk_off[b];
+  // chunked prefill: the means of the first carry[3 b + 2] blocks of this sequence were carried over from the
+  // previous chunk's workspace (pool_carry_kernel) and are not computed again
+  if (carry != nullptr && J < carry[3 * b + 2]) return;
   const int Lk = seqlens_k[b];
   const int ntok = min(kBlock, Lk - J * kBlock);
   const int chunk = threadIdx.x % CHUNKS, rg = threadIdx.x / CHUNKS;
@@ -187,6 +191,37 @@ __global__ void order_scatter_kernel(const SegInfo* __restrict__ segs, const int
   int c = count ? count[s] : segs[s].J_hi + 1;
   int pos = atomicAdd(&cursor[order_bucket(segs[s].h, c)], 1);
   order[pos] = s;
+}
+
+// ----------------------------------------------------------------------------------------
+// Pooled statistics carried from one chunk of a chunked prefill to the next (Sec. 4.3, "Compatibility with Chunked Prefill": the index stage runs once
+// per chunk; without this every chunk pools the whole cached prefix again).  The means of a block that was
+// complete in the previous chunk are the same numbers in this one: rows are copied from the previous workspace's
+// layout to this plan's.  carry[3 b + {0, 1, 2}] = first source row, first destination row, rows to copy of
+// sequence b.  grid (sequences, row groups of 8); a row of one array is Hkv x 128 elements.
+// ----------------------------------------------------------------------------------------
+__global__ void pool_carry_kernel(const int32_t* __restrict__ carry, int row_bytes16, int row_bytes8,
+                                  const uint8_t* __restrict__ s_khi, const uint8_t* __restrict__ s_klo,
+                                  const uint8_t* __restrict__ s_vbar, const uint8_t* __restrict__ s_k8hi,
+                                  const uint8_t* __restrict__ s_k8lo, uint8_t* __restrict__ d_khi,
+                                  uint8_t* __restrict__ d_klo, uint8_t* __restrict__ d_vbar,
+                                  uint8_t* __restrict__ d_k8hi, uint8_t* __restrict__ d_k8lo) {
+  const int b = blockIdx.x;
+  const int src0 = carry[3 * b], dst0 = carry[3 * b + 1], n = carry[3 * b + 2];
+  for (int j = blockIdx.y * 8; j < n; j += gridDim.y * 8) {
+    const int rows = min(8, n - j);
+    auto copy = [&](const uint8_t* s, uint8_t* d, int rb) {
+      if (rb == 0) return;
+      const uint4* sp = reinterpret_cast<const uint4*>(s + (size_t)(src0 + j) * rb);
+      uint4* dp = reinterpret_cast<uint4*>(d + (size_t)(dst0 + j) * rb);
+      for (int i = threadIdx.x; i < rows * rb / 16; i += blockDim.x) dp[i] = sp[i];
+    };
+    copy(s_khi, d_khi, row_bytes16);
+    copy(s_klo, d_klo, row_bytes16);
+    copy(s_vbar, d_vbar, row_bytes16);
+    copy(s_k8hi, d_k8hi, row_bytes8);
+    copy(s_k8lo, d_k8lo, row_bytes8);
+  }
 }
 
 }  // namespace fp2

@@ -108,3 +108,21 @@ def test_stage_calls_fail_loudly_without_a_device():
                                  None, dummy, None)
     assert code == 4            # FP2_ERR_CUDA: no kernel ran, nothing fell back to the CPU
     plan.close()
+
+
+def test_pool_carry_count_is_host_only_and_counts_complete_blocks():
+    """Blocks carried between chunks = blocks complete in both (floor(min(Lk) / 128)); needs no device."""
+    from paper_2608_19758_b200 import binding
+    def plan(seqs):
+        prm = dict(num_seqs=len(seqs), total_q=sum(l - p for l, p in seqs), num_q_heads=4, num_kv_heads=2, head_dim=128,
+                   block_size=128, tile_rows=128, page_size=16, num_pages=4096, max_pages_per_seq=1024,
+                   sink_tokens=256, window_tokens=512, use_correction=1, alpha=0.1, softmax_scale=0.0, dtype=0)
+        cu = [0]
+        for l, p in seqs:
+            cu.append(cu[-1] + l - p)
+        return binding.Plan(prm, cu, [l for l, _ in seqs])
+    src = plan([(1000, 0), (300, 0), (128, 0)])
+    dst = plan([(1500, 1000), (4000, 0), (700, 300), (129, 128)])
+    assert binding.fp2_pool_carry_count(dst, src, [0, -1, 1, 2]) == [7, 0, 2, 1]
+    with pytest.raises(binding.Fp2Error):
+        binding.fp2_pool_carry_count(dst, src, [5, -1, 1, 2])          # no such source sequence

@@ -1,4 +1,4 @@
-"""GPU parity of the index export (Algorithm 1 line 5; Sec. 4.4) against the oracle: integer work, bit-exact."""
+"""GPU parity of the index export (Algorithm 1 line 5; Sec. 3.4) against the oracle: integer work, bit-exact."""
 import numpy as np
 import pytest
 import torch

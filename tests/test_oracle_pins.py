@@ -516,7 +516,7 @@ def test_generator_density_matches_forced_fraction_on_config1():
 
 
 # ------------------------------------------------------------------------------------------
-# index export (Algorithm 1 line 5; Sec. 4.4): pinned by token coverage, by the paper's
+# index export (Algorithm 1 line 5; Sec. 3.4): pinned by token coverage, by the paper's
 # "B / 64 physical tiles per logical block" and its index-memory figure, and by the round trip
 # through Eq. 22
 # ------------------------------------------------------------------------------------------
