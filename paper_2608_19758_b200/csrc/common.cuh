@@ -34,6 +34,7 @@ struct DevParams {
   int32_t sink_blocks, window_blocks, use_correction;
   int32_t num_seqs, nseg, nblk_tot, total_q;
   int32_t fp8;
+  int32_t q_tma;     // 1: a packed query tile is a TMA box (BF16, group size divides 128): [64 elems, g heads, 128 / g tokens] x 2
   float alpha;
   float scale_log2;  // softmax scale * log2(e)
 };

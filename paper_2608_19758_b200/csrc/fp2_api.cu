@@ -220,6 +220,7 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
   d.use_correction = p->use_correction ? 1 : 0;
   d.num_seqs = p->num_seqs; d.nseg = (int32_t)pl->nseg; d.nblk_tot = (int32_t)nblk_tot; d.total_q = p->total_q;
   d.fp8 = p->dtype == FP2_FP8_E4M3;
+  d.q_tma = (!d.fp8 && 128 % g == 0) ? 1 : 0;
   d.alpha = p->alpha;
   const double sc = p->softmax_scale > 0.f ? (double)p->softmax_scale : 1.0 / sqrt((double)kHeadDim);
   d.scale_log2 = (float)(sc * 1.4426950408889634);
@@ -272,6 +273,19 @@ static bool make_map(fp2_plan* pl, CUtensorMap* m, const void* base, int64_t row
                           const_cast<void*>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// Packed query tile as a TMA box (see DevParams::q_tma): [64 elements, g heads, 128 / g tokens] of q [total_q, Hq, 128].
+static bool make_q_map(fp2_plan* pl, CUtensorMap* m, const void* q) {
+  const int g = pl->dev.group;
+  cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)pl->prm.num_q_heads, (cuuint64_t)pl->prm.total_q};
+  cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)kHeadDim * 2 * pl->prm.num_q_heads};
+  cuuint32_t box[3] = {64u, (cuuint32_t)g, (cuuint32_t)(128 / g)};
+  cuuint32_t es[3] = {1, 1, 1};
+  CUresult r = pl->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
@@ -368,14 +382,16 @@ extern "C" fp2_status fp2_select_blocks(fp2_plan* pl, const void* q, const void*
   if (!make_map(pl, &mhi, ws + pl->ws_khi, pl->nblk_tot, pl->prm.num_kv_heads, 128, false) ||
       !make_map(pl, &mlo, ws + pl->ws_klo, pl->nblk_tot, pl->prm.num_kv_heads, 128, false))
     return FP2_ERR_CUDA;
+  CUtensorMap mq = mhi;   // unused unless q_tma
+  if (pl->dev.q_tma && !make_q_map(pl, &mq, q)) return FP2_ERR_CUDA;
   int* status = reinterpret_cast<int*>(ws + pl->ws_status);
   const unsigned grid = (unsigned)(pl->nseg < pl->num_sms ? pl->nseg : pl->num_sms);
   if (pl->dev.fp8)
     score_select_kernel<true><<<grid, kScoreThreads, kScoreSmemBytes, st>>>(
-        mhi, mlo, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, status);
+        mhi, mlo, mq, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, status);
   else
     score_select_kernel<false><<<grid, kScoreThreads, kScoreSmemBytes, st>>>(
-        mhi, mlo, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, status);
+        mhi, mlo, mq, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, status);
   pl->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
@@ -386,16 +402,16 @@ extern "C" fp2_status fp2_select_blocks(fp2_plan* pl, const void* q, const void*
 // Attention: two 256-thread CTAs per SM, each a persistent worker on the shared work counter.  mkb / mkb_lo:
 // pooled keys of the correction chunks (BF16: one BF16 array, mkb_lo unused; FP8: e4m3 hi and lo).
 static void launch_attn(fp2_plan* pl, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mkb,
-                        const CUtensorMap& mkb_lo, const CUtensorMap& mvb, const AttnArgs& a, int64_t max_units,
-                        cudaStream_t st) {
+                        const CUtensorMap& mkb_lo, const CUtensorMap& mvb, const CUtensorMap& mq, const AttnArgs& a,
+                        int64_t max_units, cudaStream_t st) {
   const int64_t workers = (int64_t)pl->num_sms * AttnCfg<false>::kCtasPerSm;
   const unsigned grid = (unsigned)(max_units < workers ? max_units : workers);
   if (pl->dev.fp8)
     sparse_attn_kernel<true><<<grid, AttnCfg<true>::kThreads, AttnCfg<true>::kSmemBytes, st>>>(mk, mv, mkb, mkb_lo,
-                                                                                                 mvb, a, pl->dev);
+                                                                                                 mvb, mq, a, pl->dev);
   else
     sparse_attn_kernel<false><<<grid, AttnCfg<false>::kThreads, AttnCfg<false>::kSmemBytes, st>>>(
-        mk, mv, mkb, mkb_lo, mvb, a, pl->dev);
+        mk, mv, mkb, mkb_lo, mvb, mq, a, pl->dev);
 }
 
 static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, const void* v, const int32_t* pt,
@@ -464,7 +480,9 @@ static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, cons
     a.part_ml = reinterpret_cast<float2*>(ws + pl->ws_part_ml);
     max_units = pl->split_units_cap;
   }
-  launch_attn(pl, mk, mv, mkb, mkb_lo, mvb, a, max_units, st);
+  CUtensorMap mq = mk;   // unused unless q_tma
+  if (pl->dev.q_tma && !make_q_map(pl, &mq, q)) return FP2_ERR_CUDA;
+  launch_attn(pl, mk, mv, mkb, mkb_lo, mvb, mq, a, max_units, st);
   pl->last_launches += 1;
   if (split) {
     int32_t* seg_split = reinterpret_cast<int32_t*>(ws + pl->ws_seg_split);
@@ -570,7 +588,9 @@ extern "C" fp2_status fp2_dense_prefill_static(fp2_plan* pl, const void* q, cons
   a.status = reinterpret_cast<int*>(sw);
   // the dense path stages no pooled chunks: the two pooled-mean maps are never dereferenced
   a.unit_split = nullptr; a.n_units = nullptr; a.part_o = nullptr; a.part_ml = nullptr;
-  launch_attn(pl, mk, mv, mk, mk, mv, a, pl->nseg, st);
+  CUtensorMap mq = mk;   // unused unless q_tma
+  if (pl->dev.q_tma && !make_q_map(pl, &mq, q)) return FP2_ERR_CUDA;
+  launch_attn(pl, mk, mv, mk, mk, mv, mq, a, pl->nseg, st);
   pl->last_launches = 4;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }

@@ -208,7 +208,7 @@ __device__ __forceinline__ void load_q_tile_async(uint8_t* sQ, const uint8_t* __
 template <bool FP8>
 __global__ void __launch_bounds__(kScoreThreads, 1)
 score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_constant__ CUtensorMap map_klo,
-                    const uint8_t* __restrict__ q, const SegInfo* __restrict__ segs, const float* __restrict__ q_scale,
+                    const __grid_constant__ CUtensorMap map_q, const uint8_t* __restrict__ q, const SegInfo* __restrict__ segs, const float* __restrict__ q_scale,
                     DevParams P, int64_t* __restrict__ seg_offset, int32_t* __restrict__ seg_count,
                     int32_t* __restrict__ blk_idx, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
@@ -291,6 +291,37 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       cp_async_commit();
       return true;
     };
+    if (!FP8 && P.q_tma) {
+      // Under PackGQA (Eq. 13) packed row r is (token r / g, head r % g): when g divides 128 a tile is 128 / g
+      // consecutive tokens x g consecutive heads, i.e. one TMA box per 64-element half, landing in exactly the
+      // swizzled layout the MMA reads.  No thread touches the data; the tile's barrier carries the byte count.
+      // Rows past the end of a short last tile read the tokens that follow (or zeros past the tensor's end) and are
+      // never used.  Three tiles in flight.
+      const uint64_t pol = l2_policy_evict_first();
+      for (int k = 0;; ++k) {
+        const int slot = k % kScoreInfoSlots, qb = k % kScoreQBufs;
+        if (k >= kScoreInfoSlots) mbar_wait(&info_empty[slot], ((k / kScoreInfoSlots) - 1) & 1, ctx, 111);
+        const int sgi = seg_of(k);
+        const bool valid = sgi >= 0;
+        if (t64 == 0) {
+          info_valid[slot] = valid;
+          if (valid) info[slot] = segs[sgi];
+        }
+        named_bar_sync(2, 64);
+        if (t64 == 0) mbar_arrive(&info_full[slot]);
+        if (!valid) break;
+        if (k >= kScoreQBufs) mbar_wait(&q_empty[qb], ((k / kScoreQBufs) - 1) & 1, ctx, 112);
+        if (t64 == 0) {
+          const SegInfo& sg = info[slot];
+          uint8_t* dst = sQ + qb * 32768;
+          mbar_arrive_expect_tx(&q_full[qb], 32768);
+          tma_load_3d_hint(dst, &map_q, &q_full[qb], 0, sg.h * P.group, sg.q_tok0 + sg.r0 / P.group, pol);
+          tma_load_3d_hint(dst + 16384, &map_q, &q_full[qb], 64, sg.h * P.group, sg.q_tok0 + sg.r0 / P.group, pol);
+        } else {
+          mbar_arrive(&q_full[qb]);
+        }
+      }
+    } else {
     bool have = issue(0);
     for (int k = 0; have; ++k) {
       const bool next = issue(k + 1);
@@ -307,6 +338,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       fence_proxy_async();
       mbar_arrive(&q_full[qb]);
       have = next;
+    }
     }
   } else if (warp == 8) {
     // ---------------- producer: kbar pieces (hi, lo of every 128-block chunk) via TMA ----------------

@@ -179,12 +179,13 @@ __device__ __forceinline__ float row_exp(const uint32_t (&x)[128], uint32_t p_ad
 }
 
 // map_kbar / map_kbar_lo: pooled keys of the correction chunks -- BF16: one BF16 array (map_kbar_lo unused);
-// FP8: the e4m3 hi and lo arrays.  map_vbar: pooled values, 16-bit.
+// FP8: the e4m3 hi and lo arrays.  map_vbar: pooled values, 16-bit.  map_q: packed query tiles (DevParams::q_tma).
 template <bool FP8>
 __global__ void __launch_bounds__(AttnCfg<FP8>::kThreads, AttnCfg<FP8>::kCtasPerSm)
 sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v,
                     const __grid_constant__ CUtensorMap map_kbar, const __grid_constant__ CUtensorMap map_kbar_lo,
-                    const __grid_constant__ CUtensorMap map_vbar, AttnArgs A, DevParams P) {
+                    const __grid_constant__ CUtensorMap map_vbar, const __grid_constant__ CUtensorMap map_q,
+                    AttnArgs A, DevParams P) {
   constexpr int kSetupThreads = 64;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -332,6 +333,20 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       if (!valid) break;
       // Q tile: wait until every S = Q K^T of the previous unit has completed, then overwrite
       if (it >= 1) mbar_wait(&q_empty, (it - 1) & 1, ctx, 202);
+      if (!FP8 && P.q_tma) {
+        // PackGQA (Eq. 13) with a group size that divides 128: the tile is 128 / g tokens x g heads, one TMA box
+        // per 64-element half, landing in the swizzled layout the MMA reads
+        if (t64 == 0) {
+          const SegInfo& sg = ti.sg;
+          const uint64_t pol = l2_policy_evict_first();
+          mbar_arrive_expect_tx(&q_full, kTileBytes);
+          tma_load_3d_hint(sQ, &map_q, &q_full, 0, sg.h * g, sg.q_tok0 + sg.r0 / g, pol);
+          tma_load_3d_hint(sQ + 16384, &map_q, &q_full, 64, sg.h * g, sg.q_tok0 + sg.r0 / g, pol);
+        } else {
+          mbar_arrive(&q_full);
+        }
+        continue;
+      }
       if constexpr (FP8) {
         load_q_raw_async(sQ, A.q, ti.sg, P, t64, kSetupThreads);
         cp_async_wait_all();
