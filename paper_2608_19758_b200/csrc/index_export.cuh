@@ -47,26 +47,51 @@ __global__ void csr_count_kernel(const SegInfo* __restrict__ segs, const int32_t
   cu[g + 1] = n;
 }
 
-// single CTA of 1024 threads: inclusive scan of cu[1 .. n] in place (cu[g + 1] = tiles of segments 0..g)
-__global__ void csr_scan_kernel(int32_t* __restrict__ cu, int n) {
-  __shared__ int32_t part[1024];
+// single CTA of 1024 threads: inclusive scan of cu[1 .. n] in place (cu[g + 1] = tiles of segments 0..g).
+// Tiles of kScanTile = 1024 x 8 elements: every thread loads its 8 consecutive values at once, scans them in
+// registers, the CTA scans the 1024 thread totals through shared memory, and a running carry links the tiles.
+constexpr int kScanPerThread = 8;
+__global__ void __launch_bounds__(1024, 1) csr_scan_kernel(int32_t* __restrict__ cu, int n) {
+  __shared__ int32_t warp_tot[32];
+  __shared__ int32_t s_carry;
   int32_t* v = cu + 1;
-  const int per = (n + 1023) / 1024;
-  const int beg = threadIdx.x * per, end = min(beg + per, n);
-  int s = 0;
-  for (int i = beg; i < end; ++i) s += v[i];
-  part[threadIdx.x] = s;
+  const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+  if (t == 0) s_carry = 0;
   __syncthreads();
-  for (int d = 1; d < 1024; d <<= 1) {
-    const int add = threadIdx.x >= d ? part[threadIdx.x - d] : 0;
+  for (int base = 0; base < n; base += 1024 * kScanPerThread) {
+    const int i0 = base + t * kScanPerThread;
+    int32_t x[kScanPerThread];
+#pragma unroll
+    for (int j = 0; j < kScanPerThread; ++j) x[j] = i0 + j < n ? v[i0 + j] : 0;
+#pragma unroll
+    for (int j = 1; j < kScanPerThread; ++j) x[j] += x[j - 1];
+    // exclusive prefix of the thread totals: warp scan, then the 32 warp totals
+    int32_t incl = x[kScanPerThread - 1];
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int32_t y = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += y;
+    }
+    if (lane == 31) warp_tot[w] = incl;
     __syncthreads();
-    part[threadIdx.x] += add;
+    if (w == 0) {
+      int32_t wt = warp_tot[lane];
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int32_t y = __shfl_up_sync(0xffffffffu, wt, d);
+        if (lane >= d) wt += y;
+      }
+      warp_tot[lane] = wt;   // inclusive over warps
+    }
     __syncthreads();
-  }
-  int run = part[threadIdx.x] - s;
-  for (int i = beg; i < end; ++i) {
-    run += v[i];
-    v[i] = run;
+    const int32_t carry = s_carry;
+    const int32_t before = carry + (w > 0 ? warp_tot[w - 1] : 0) + incl - x[kScanPerThread - 1];
+#pragma unroll
+    for (int j = 0; j < kScanPerThread; ++j)
+      if (i0 + j < n) v[i0 + j] = x[j] + before;
+    __syncthreads();
+    if (t == 1023) s_carry = carry + warp_tot[31];
+    __syncthreads();
   }
 }
 
