@@ -176,8 +176,10 @@ def main():
             return
         case = inputs.make_case(spec)
         times, fl = [], 0.0
+        # about 600 segments over the whole run (a few minutes of host time), at most 48 per step
+        per_step = max(4, min(48, 600 // (args.warmup + args.steps)))
         for i in range(args.warmup + args.steps):
-            dt, fl, desc, threads = oracle_sample(case, max(4, args.oracle_segments // 4), seed=i)
+            dt, fl, desc, threads = oracle_sample(case, per_step, seed=i)
             if i >= args.warmup:
                 times.append(dt)
         ms = 1e3 * float(np.mean(times))
