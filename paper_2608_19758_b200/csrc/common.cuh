@@ -34,7 +34,8 @@ struct DevParams {
   int32_t sink_blocks, window_blocks, use_correction;
   int32_t num_seqs, nseg, nblk_tot, total_q;
   int32_t fp8;
-  int32_t q_tma;     // 1: a packed query tile is a TMA box (BF16, group size divides 128): [64 elems, g heads, 128 / g tokens] x 2
+  int32_t q_tma;     // 1: the group size divides 128, so a packed query tile is a TMA box [128 bytes, g heads, 128 / g tokens]
+                     //    (x 2 for BF16); used by the attention kernel (both dtypes) and the BF16 scorer
   float alpha;
   float scale_log2;  // softmax scale * log2(e)
 };

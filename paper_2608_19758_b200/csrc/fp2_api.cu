@@ -220,7 +220,7 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
   d.use_correction = p->use_correction ? 1 : 0;
   d.num_seqs = p->num_seqs; d.nseg = (int32_t)pl->nseg; d.nblk_tot = (int32_t)nblk_tot; d.total_q = p->total_q;
   d.fp8 = p->dtype == FP2_FP8_E4M3;
-  d.q_tma = (!d.fp8 && 128 % g == 0) ? 1 : 0;
+  d.q_tma = (128 % g == 0) ? 1 : 0;
   d.alpha = p->alpha;
   const double sc = p->softmax_scale > 0.f ? (double)p->softmax_scale : 1.0 / sqrt((double)kHeadDim);
   d.scale_log2 = (float)(sc * 1.4426950408889634);
@@ -276,16 +276,20 @@ static bool make_map(fp2_plan* pl, CUtensorMap* m, const void* base, int64_t row
   return r == CUDA_SUCCESS;
 }
 
-// Packed query tile as a TMA box (see DevParams::q_tma): [64 elements, g heads, 128 / g tokens] of q [total_q, Hq, 128].
+// Packed query tile as a TMA box (see DevParams::q_tma): [128 bytes, g heads, 128 / g tokens] of q [total_q, Hq, 128]
+// -- 64 BF16 elements (the tile takes two boxes) or 128 e4m3 bytes (one box).
 static bool make_q_map(fp2_plan* pl, CUtensorMap* m, const void* q) {
   const int g = pl->dev.group;
+  const bool fp8 = pl->dev.fp8;
+  const cuuint64_t esz = fp8 ? 1 : 2;
   cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)pl->prm.num_q_heads, (cuuint64_t)pl->prm.total_q};
-  cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)kHeadDim * 2 * pl->prm.num_q_heads};
-  cuuint32_t box[3] = {64u, (cuuint32_t)g, (cuuint32_t)(128 / g)};
+  cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * esz, (cuuint64_t)kHeadDim * esz * pl->prm.num_q_heads};
+  cuuint32_t box[3] = {fp8 ? 128u : 64u, (cuuint32_t)g, (cuuint32_t)(128 / g)};
   cuuint32_t es[3] = {1, 1, 1};
-  CUresult r = pl->encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box, es,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  CUresult r = pl->encode(m, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+                          const_cast<void*>(q), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 

@@ -333,15 +333,17 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       if (!valid) break;
       // Q tile: wait until every S = Q K^T of the previous unit has completed, then overwrite
       if (it >= 1) mbar_wait(&q_empty, (it - 1) & 1, ctx, 202);
-      if (!FP8 && P.q_tma) {
+      if (P.q_tma) {
         // PackGQA (Eq. 13) with a group size that divides 128: the tile is 128 / g tokens x g heads, one TMA box
-        // per 64-element half, landing in the swizzled layout the MMA reads
+        // per 128 bytes of a row (two 64-element halves for BF16, the whole row for e4m3), landing in the swizzled
+        // layout the MMA reads.  Rows past the end of a short last tile get whatever follows; nothing reads them.
         if (t64 == 0) {
           const SegInfo& sg = ti.sg;
           const uint64_t pol = l2_policy_evict_first();
-          mbar_arrive_expect_tx(&q_full, kTileBytes);
+          mbar_arrive_expect_tx(&q_full, FP8 ? kRawBytes : kTileBytes);
           tma_load_3d_hint(sQ, &map_q, &q_full, 0, sg.h * g, sg.q_tok0 + sg.r0 / g, pol);
-          tma_load_3d_hint(sQ + 16384, &map_q, &q_full, 64, sg.h * g, sg.q_tok0 + sg.r0 / g, pol);
+          if constexpr (!FP8)
+            tma_load_3d_hint(sQ + 16384, &map_q, &q_full, 64, sg.h * g, sg.q_tok0 + sg.r0 / g, pol);
         } else {
           mbar_arrive(&q_full);
         }
