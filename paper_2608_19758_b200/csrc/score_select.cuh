@@ -14,10 +14,11 @@
 // relative; a single BF16 kbar would move them by ~3e-3 and flip list entries.  FP8 inputs: the query tile is
 // widened to F16 (exact) and kbar is an F16 (hi, lo) pair.
 //
-// Roles: warps 0-3 / 4-7 = two consumer warpgroups alternating over chunks (TMEM accumulators 0 / 1) and doing
-// the selection of their tile together; warp 8 = TMA producer of kbar pieces; warp 9 = UMMA issuer; warps 10-11
-// fetch the next segment and stage its query tile into the free one of two Q buffers, so that the next tile's
-// MMAs start while the current tile is still being exponentiated and selected.
+// Roles: warps 0-3 / 4-7 = two consumer warpgroups alternating over chunks (TMEM accumulators 0 / 1); warp 8 = TMA
+// producer of kbar pieces; warp 9 = UMMA issuer; warps 10-11 fetch the next segment and stage its query tile into
+// a free Q buffer, so that the next tile's MMAs start while the current tile is still being exponentiated.
+// Selection: by the consumers together at the end of their tile -- or, when the query tiles come by TMA (BF16,
+// group size divides 128) and warp 10 alone can feed them, by warp 11 beside the scoring of the next tile.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
@@ -226,21 +227,33 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
   __shared__ uint64_t full[kScoreStages], empty[kScoreStages], acc_full[2], acc_empty[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
-  __shared__ float red[8];
+  __shared__ float red[2][8];
   __shared__ int wsum[8];
+  __shared__ uint64_t e_full[2], sel_done[2];   // async mode: [tile & 1] energies of the tile are complete / its list is written
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   WaitCtx ctx{status, &abort_flag};
+  // When the query tiles come by TMA, one set-up warp is enough and the other (warp 11) takes the selection off
+  // the consumers: they only leave the tile's energies (and their maxima) in shared memory and go on with the next
+  // tile's chunks; threshold, forced blocks and the ordered compaction of tile t run beside the scoring of tile
+  // t+1.  The energy buffer is used in two halves by tile parity; a tile with more than kMaxBlocks / 2 candidates
+  // takes both and waits for its neighbours.  In this mode the two warpgroups also share the chunks by a count
+  // that runs across tiles, so a tile with an odd number of chunks leaves neither of them short.
+  const bool async_sel = !FP8 && P.q_tma;
 
   if (tid == 0) {
     abort_flag = 0;
     for (int i = 0; i < kScoreInfoSlots; ++i) {
       mbar_init(&info_full[i], 1);
-      mbar_init(&info_empty[i], 2 + 256);
+      mbar_init(&info_empty[i], 2 + 256 + (async_sel ? 1 : 0));   // producer, issuer, consumers (, selection warp)
     }
     for (int i = 0; i < kScoreQBufs; ++i) {
-      mbar_init(&q_full[i], 64);
+      mbar_init(&q_full[i], async_sel ? 1 : 64);
       mbar_init(&q_empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&e_full[i], 256);
+      mbar_init(&sel_done[i], 1);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&acc_full[i], 1);
@@ -261,8 +274,8 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
 
-  if (warp >= 10) {
-    // ---------------- set-up: segment k of this CTA is number blockIdx.x + k * gridDim.x in heaviest-first order
+  if (warp == 10 || (warp == 11 && !async_sel)) {
+    // ---------------- set-up (warps 10 and 11; warp 10 alone when the tiles come by TMA): segment k of this CTA is number blockIdx.x + k * gridDim.x in heaviest-first order
     // (a static round-robin: no atomic on the critical path).  The loop is software-pipelined: the copies of
     // tile k+1 are issued before the copies of tile k are waited for, so two query tiles are in flight.
     const int t64 = tid - 320;
@@ -291,7 +304,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       cp_async_commit();
       return true;
     };
-    if (!FP8 && P.q_tma) {
+    if (async_sel) {
       // Under PackGQA (Eq. 13) packed row r is (token r / g, head r % g): when g divides 128 a tile is 128 / g
       // consecutive tokens x g consecutive heads, i.e. one TMA box per 64-element half, landing in exactly the
       // swizzled layout the MMA reads.  No thread touches the data; the tile's barrier carries the byte count.
@@ -306,9 +319,10 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
         if (t64 == 0) {
           info_valid[slot] = valid;
           if (valid) info[slot] = segs[sgi];
+          __threadfence_block();
+          mbar_arrive(&info_full[slot]);
         }
-        named_bar_sync(2, 64);
-        if (t64 == 0) mbar_arrive(&info_full[slot]);
+        __syncwarp();
         if (!valid) break;
         if (k >= kScoreQBufs) mbar_wait(&q_empty[qb], ((k / kScoreQBufs) - 1) & 1, ctx, 112);
         if (t64 == 0) {
@@ -317,9 +331,8 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
           mbar_arrive_expect_tx(&q_full[qb], 32768);
           tma_load_3d_hint(dst, &map_q, &q_full[qb], 0, sg.h * P.group, sg.q_tok0 + sg.r0 / P.group, pol);
           tma_load_3d_hint(dst + 16384, &map_q, &q_full[qb], 64, sg.h * P.group, sg.q_tok0 + sg.r0 / P.group, pol);
-        } else {
-          mbar_arrive(&q_full[qb]);
         }
+        __syncwarp();
       }
     } else {
     bool have = issue(0);
@@ -339,6 +352,39 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       mbar_arrive(&q_full[qb]);
       have = next;
     }
+    }
+  } else if (warp == 11) {
+    // ---------------- selection warp (async mode): threshold, forced blocks, ordered compaction of tile `it` ----------------
+    for (int it = 0;; ++it) {
+      const int slot = it % kScoreInfoSlots, eb = it & 1;
+      mbar_wait(&info_full[slot], (it / kScoreInfoSlots) & 1, ctx, 151);
+      if (!info_valid[slot]) break;
+      const SegInfo sg = info[slot];
+      const int ncand = sg.J_hi + 1;
+      const float* e = sE + (ncand > kMaxBlocks / 2 ? 0 : eb * (kMaxBlocks / 2));
+      mbar_wait(&e_full[eb], (it >> 1) & 1, ctx, 152);
+      float maxE = red[eb][0];
+#pragma unroll
+      for (int i = 1; i < 8; ++i) maxE = fmaxf(maxE, red[eb][i]);
+      // J selected  <=>  E_J >= alpha max E  <=>  e_J >= log2(alpha) + max e   (alpha <= 0 selects everything)
+      const float thr = P.alpha > 0.f ? maxE + log2f(P.alpha) : -INFINITY;
+      const int win_lo = sg.J_lo - P.window_blocks;
+      int pos = 0;
+      for (int J0 = 0; J0 < ncand; J0 += 32) {
+        const int J = J0 + lane;
+        const bool keep = J < ncand && (e[J] >= thr || J < P.sink_blocks || J >= win_lo);
+        const unsigned bal = __ballot_sync(0xffffffffu, keep);
+        if (keep) blk_idx[sg.off + pos + __popc(bal & ((1u << lane) - 1u))] = J;
+        pos += __popc(bal);
+      }
+      __syncwarp();
+      if (lane == 0) {
+        seg_count[sg.seg] = pos;
+        seg_offset[sg.seg] = sg.off;
+        if (sg.seg == P.nseg - 1) seg_offset[P.nseg] = sg.off + ncand;
+        mbar_arrive(&sel_done[eb]);
+        mbar_arrive(&info_empty[slot]);
+      }
     }
   } else if (warp == 8) {
     // ---------------- producer: kbar pieces (hi, lo of every 128-block chunk) via TMA ----------------
@@ -372,7 +418,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
     // ---------------- UMMA issuer: acc[c & 1] = kbar_hi Q^T + kbar_lo Q^T ----------------
     if (lane == 0) {
       constexpr uint32_t idesc = FP8 ? make_idesc(128, 128, 0, 0, 0, 0) : make_idesc(128, 128, 1, 1, 0, 0);
-      uint32_t pc = 0, ac0 = 0, ac1 = 0;
+      uint32_t pc = 0, ac0 = 0, ac1 = 0, gc0 = 0;   // gc0: chunks of all earlier tiles (async mode), else 0
       for (int it = 0;; ++it) {
         const int slot = it % kScoreInfoSlots, qb = it % kScoreQBufs;
         mbar_wait(&info_full[slot], (it / kScoreInfoSlots) & 1, ctx, 131);
@@ -381,7 +427,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
         mbar_wait(&q_full[qb], (it / kScoreQBufs) & 1, ctx, 132);
         const uint32_t q_addr = smem_u32(sQ + qb * 32768);
         for (int c = 0; c < nchunks; ++c) {
-          const int a = c & 1;
+          const int a = (gc0 + c) & 1;
           uint32_t& ac = a ? ac1 : ac0;
           if (ac >= 1) mbar_wait(&acc_empty[a], (ac - 1) & 1, ctx, 133);
           ++ac;
@@ -404,6 +450,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
         }
         umma_commit(&q_empty[qb]);
         mbar_arrive(&info_empty[slot]);
+        if (async_sel) gc0 += nchunks;
       }
     }
   } else {
@@ -413,6 +460,8 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
     const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + wg * 128;
     const float cs = P.scale_log2;
     uint32_t uc = 0;  // uses of this warpgroup's accumulator
+    uint32_t gc0 = 0;  // chunks of all earlier tiles (async mode), else 0
+    bool prev_big = false;
     for (int it = 0;; ++it) {
       const int slot = it % kScoreInfoSlots, qb = it % kScoreQBufs;
       mbar_wait(&info_full[slot], (it / kScoreInfoSlots) & 1, ctx, 141);
@@ -424,7 +473,17 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       // per candidate: log2 of its energy, e_J = m_J + log2(S_J)  (Eq. 1-2 / Eq. 20 in the log domain: the
       // common factor 2^-M of Eq. 20 cancels in the comparison with alpha * max)
       float lmax = -INFINITY;
-      for (int c = wg; c < nchunks; c += 2, ++uc) {
+      const int eb = it & 1;
+      const bool big = ncand > kMaxBlocks / 2;
+      float* e_out = sE + ((async_sel && !big) ? eb * (kMaxBlocks / 2) : 0);
+      if (async_sel) {
+        // the half of the energy buffer this tile writes must have been read by the selection of tile it-2, and a
+        // tile that takes (or follows one that took) the whole buffer also waits for tile it-1
+        if (it >= 2) mbar_wait(&sel_done[eb], ((it >> 1) - 1) & 1, ctx, 143);
+        if (it >= 1 && (big || prev_big)) mbar_wait(&sel_done[eb ^ 1], ((it - 1) >> 1) & 1, ctx, 144);
+        prev_big = big;
+      }
+      for (int c = (int)((gc0 ^ (uint32_t)wg) & 1u); c < nchunks; c += 2, ++uc) {
         mbar_wait(&acc_full[wg], uc & 1, ctx, 142);
         tc_fence_after();
         float m, sum;
@@ -433,18 +492,27 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
         const int J = c * 128 + key;
         if (J < ncand) {
           const float e = m + log2f(sum);
-          sE[J] = e;
+          e_out[J] = e;
           lmax = fmaxf(lmax, e);
         }
       }
-      // ---------------- selection: all 256 consumer threads, three barriers per tile ----------------
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) lmax = fmaxf(lmax, __shfl_xor_sync(0xffffffffu, lmax, o));
-      if (lane == 0) red[warp] = lmax;
+      if (async_sel) {
+        // hand the tile to the selection warp and go on
+        if (lane == 0) red[eb][warp] = lmax;
+        __syncwarp();
+        mbar_arrive(&e_full[eb]);
+        mbar_arrive(&info_empty[slot]);
+        gc0 += (uint32_t)nchunks;
+        continue;
+      }
+      // ---------------- selection: all 256 consumer threads, three barriers per tile ----------------
+      if (lane == 0) red[0][warp] = lmax;
       named_bar_sync(1, 256);            // energies and per-warp maxima are visible
-      float maxE = red[0];
+      float maxE = red[0][0];
 #pragma unroll
-      for (int i = 1; i < 8; ++i) maxE = fmaxf(maxE, red[i]);
+      for (int i = 1; i < 8; ++i) maxE = fmaxf(maxE, red[0][i]);
       // J selected  <=>  E_J >= alpha max E  <=>  e_J >= log2(alpha) + max e   (alpha <= 0 selects everything)
       const float thr = P.alpha > 0.f ? maxE + log2f(P.alpha) : -INFINITY;
       const int win_lo = sg.J_lo - P.window_blocks;
