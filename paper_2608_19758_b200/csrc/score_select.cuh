@@ -147,13 +147,19 @@ __device__ __forceinline__ void score_chunk(uint32_t lane_addr, float cs, const 
   tmem_wait_ld();
   tc_fence_before();
   mbar_arrive(acc_empty_bar);
-  // x_j = s_j * multiplier (packed fp32x2), rows past nrows masked to -inf
+  // x_j = s_j * multiplier, rows past nrows masked to -inf.  BF16: one multiplier for all rows, which commutes
+  // with the maximum (it is positive): the maximum is taken over the raw logits and the scaling rides in the
+  // fused multiply-add that subtracts it.  FP8: a multiplier per row (q_scale), applied first.
   float x[128];
 #pragma unroll
   for (int j = 0; j < 128; j += 2) {
-    uint64_t mult2 = f2_pack(cs, cs);
-    if constexpr (FP8) mult2 = f2_pack(sC[j], sC[j + 1]);
-    f2_unpack(f2_mul(f2_pack(__uint_as_float(xv[j]), __uint_as_float(xv[j + 1])), mult2), x[j], x[j + 1]);
+    if constexpr (FP8) {
+      const uint64_t mult2 = f2_pack(sC[j], sC[j + 1]);
+      f2_unpack(f2_mul(f2_pack(__uint_as_float(xv[j]), __uint_as_float(xv[j + 1])), mult2), x[j], x[j + 1]);
+    } else {
+      x[j] = __uint_as_float(xv[j]);
+      x[j + 1] = __uint_as_float(xv[j + 1]);
+    }
     if constexpr (PARTIAL) {
       x[j] = (j < nrows) ? x[j] : -INFINITY;
       x[j + 1] = (j + 1 < nrows) ? x[j + 1] : -INFINITY;
@@ -166,13 +172,16 @@ __device__ __forceinline__ void score_chunk(uint32_t lane_addr, float cs, const 
     m8[c] = max3(max3(max3(v[0], v[1], v[2]), max3(v[3], v[4], v[5]), max3(v[6], v[7], v[8])),
                  max3(v[9], v[10], v[11]), max3(max3(v[12], v[13], v[14]), v[15], v[15]));
   }
-  const float m = fmaxf(max3(m8[0], m8[1], m8[2]), max3(max3(m8[3], m8[4], m8[5]), m8[6], m8[7]));
-  const uint64_t nm2 = f2_pack(-m, -m);
+  float m = fmaxf(max3(m8[0], m8[1], m8[2]), max3(max3(m8[3], m8[4], m8[5]), m8[6], m8[7]));
+  const float mul = FP8 ? 1.0f : cs;
+  m *= mul;
+  const uint64_t nm2 = f2_pack(-m, -m), mul2 = f2_pack(mul, mul);
   uint64_t s4[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
   for (int j = 0; j < 128; j += 2) {
     float d0, d1;
-    f2_unpack(f2_add(f2_pack(x[j], x[j + 1]), nm2), d0, d1);
+    if constexpr (FP8) f2_unpack(f2_add(f2_pack(x[j], x[j + 1]), nm2), d0, d1);
+    else f2_unpack(f2_fma(f2_pack(x[j], x[j + 1]), mul2, nm2), d0, d1);
     s4[(j >> 1) & 3] = f2_add(s4[(j >> 1) & 3], f2_pack(ex2(d0), ex2(d1)));
   }
   float t0, t1;
