@@ -457,10 +457,10 @@ def main():
     if rank != 0:
         return
     # DRAM bytes per attention launch (dram__bytes_read.sum + dram__bytes_write.sum, one ncu pass on the full
-    # workload, profiles/bench_config3_launch_list.md): 3.30 GB read + 1.06 GB written at config 3 / 95 % sparsity,
+    # workload, profiles/bench_config3_launch_list.md): 3.29 GB read + 1.06 GB written at config 3 / 95 % sparsity,
     # against 1.07 (Q) + 0.54 (K, V) + 1.07 (O) GB algorithmic: K/V pages are re-read from DRAM about four times
     # because one KV head's 67 MB working set does not stay resident in L2 next to the streaming Q / O traffic.
-    traffic = 4.36e9 if (args.config == 3 and args.scale_down == 1 and abs(args.sparsity - 0.95) < 1e-6) else None
+    traffic = 4.35e9 if (args.config == 3 and args.scale_down == 1 and abs(args.sparsity - 0.95) < 1e-6) else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
