@@ -256,6 +256,27 @@ def test_ragged_and_degenerate_batches(seqs):
     full_pipeline(spec)
 
 
+def test_tiles_with_more_candidates_than_half_the_energy_buffer():
+    """The scorer keeps the energies of two consecutive tiles in two halves of one buffer while a separate warp
+    selects; a tile with more than 2048 candidate blocks (a sequence beyond 256K tokens) takes the whole buffer
+    and must wait for both neighbours.  A chunk of 4096 new tokens behind a 262144-token prefix gives 32 such
+    tiles; the short sequences around it give ordinary tiles before and after."""
+    spec = inputs.small_spec(seqs=[(700, 0), (266240, 262144), (1000, 0)], num_q_heads=1, num_kv_heads=1,
+                             page_size=64, config_id=61)
+    spec.alpha = 0.02
+    case, dc, wl = make(spec)
+    for _ in range(2):   # twice: the second run starts from whatever the first left in shared structures
+        dc.select()
+        dc.status()
+        tot, near = check_lists(dc, wl)
+    big = [s for s in wl.segs if s.J_hi + 1 > 2048]
+    assert len(big) == 32 and len(wl.segs) > 40
+    lists = dc.lists_host()
+    dc.sparse()
+    dc.status()
+    check_attention(dc, wl, lists, dtype=spec.dtype)
+
+
 @pytest.mark.parametrize("alpha", [0.0, 2.0, 1.0])
 def test_alpha_extremes(alpha):
     spec = inputs.small_spec(seqs=[(2000, 0)], num_q_heads=4, num_kv_heads=1, page_size=64, config_id=81, sink=False)
