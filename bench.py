@@ -61,7 +61,7 @@ class ClockSampler:
            "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap",
            "--format=csv,noheader,nounits", "-lms", "50"]
 
-    def __init__(self, gpu_index: int):
+    def __init__(self, gpu_index):
         self.gpu = gpu_index
         self.lines = []
         self.proc = None
@@ -84,7 +84,7 @@ class ClockSampler:
         sm, mx, reasons = [], [], set()
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
-            if len(f) < 9 or not f[0].isdigit() or int(f[0]) != self.gpu:
+            if len(f) < 9 or not f[0].isdigit():   # nvidia-smi was asked for this GPU only (-i)
                 continue
             try:
                 sm.append(float(f[1])); mx.append(float(f[2]))
@@ -98,13 +98,13 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def physical_gpu_index(local: int) -> int:
+def physical_gpu_index(local: int):
+    """What `nvidia-smi -i` should be given for this rank's device: an index, or the UUID CUDA_VISIBLE_DEVICES names."""
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
-        try:
-            return int(vis.split(",")[local])
-        except Exception:
-            return local
+        ids = [x.strip() for x in vis.split(",") if x.strip()]
+        if local < len(ids):
+            return int(ids[local]) if ids[local].isdigit() else ids[local]
     return local
 
 
