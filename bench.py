@@ -81,7 +81,7 @@ class ClockSampler:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
-        sm, mx, reasons = [], [], set()
+        sm, mx, reasons, masks = [], [], set(), set()
         for ln in self.lines:
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 9 or not f[0].isdigit():   # nvidia-smi was asked for this GPU only (-i)
@@ -90,12 +90,13 @@ class ClockSampler:
                 sm.append(float(f[1])); mx.append(float(f[2]))
             except ValueError:
                 continue
+            masks.add(f[4])   # clocks_event_reasons.active, the raw bit mask
             for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
                 if val.lower().startswith("active"):
                     reasons.add(name)
         busy = [x for x in sm if x > 0]
         return {"sm_mhz": float(np.median(busy)) if busy else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "reason_masks": sorted(masks)}
 
 
 def physical_gpu_index(local: int):
