@@ -31,10 +31,16 @@
  *     exclusive scan of ntiles.  Lists are a padded CSR: seg_offset[seg] (fixed by the plan: exclusive scan
  *     of the candidate counts J_hi + 1), seg_count[seg] selected blocks, blk_idx[seg_offset[seg] + k]
  *     ascending ids of 128-token KV blocks.
+ *   - Lengths.  Every kernel takes its geometry (lengths, prefixes, tiles, block ranges) from the plan, i.e. from
+ *     the HOST copies given to fp2_plan_create, which are validated there.  The device arrays cu_seqlens_q and
+ *     seqlens_k of the stage calls must hold the same values; the current kernels do not read them, so a
+ *     disagreement cannot move an access out of bounds.
  *   - Errors.  Every call returns an fp2_status.  Problems visible on the host (null pointers, unsupported
- *     shapes, lengths that disagree with the plan) are reported before anything is launched.  The device
- *     never traps: waits inside the kernels are bounded and list entries are clamped; both conditions are
- *     recorded in a status block that fp2_read_status returns.
+ *     shapes, inconsistent lengths in fp2_plan_create) are reported before anything is launched.  The device
+ *     never traps: waits inside the kernels are bounded; list entries outside 0..J_hi are clamped; a page id
+ *     outside [0, num_pages) in a live page-table entry is not dereferenced (pooling reads zeros for its tokens,
+ *     the attention kernel skips the page).  Each of these conditions is recorded in a status block that
+ *     fp2_read_status returns.
  */
 #ifndef FP2_H_
 #define FP2_H_
@@ -110,6 +116,16 @@ fp2_status fp2_select_blocks(fp2_plan* plan, const void* q, const void* k_cache,
                              int64_t* seg_offset, int32_t* seg_count, int32_t* blk_idx, void* workspace,
                              fp2_stream stream);
 
+/* Block-mean pooling alone (Eq. 5; Algorithm 1 line 2): the first kernel of fp2_select_blocks as a call of its own.
+ * Reads K and V once through the page table and leaves the per-block means (kbar, vbar of every 128-token block
+ * and KV head, in the operand formats the scorer and the correction chunks read) in `workspace`, exactly as
+ * fp2_select_blocks does.  For callers that refresh the pooled statistics without re-running the selection (lists
+ * supplied by the caller, then fp2_sparse_prefill with pooled_valid = 1), and for timing the pooling pass by
+ * itself.  k_scale / v_scale are read for FP8 plans only.  One kernel on `stream`; nothing is allocated. */
+fp2_status fp2_pool_blocks(fp2_plan* plan, const void* k_cache, const void* v_cache, const int32_t* page_table,
+                           const int32_t* seqlens_k, const float* k_scale, const float* v_scale, void* workspace,
+                           fp2_stream stream);
+
 /* Stage 2 (Algorithm 1, lines 6-11; Eq. 4, Eq. 6).  Attends exactly over the listed blocks; with
  * use_correction = 1 every unlisted block J < J_lo (fully visible to the whole tile) contributes
  * |B_J| e^{q.kbar_J / sqrt(d)} (vbar_J, 1) to numerator and denominator.  The lists may come from
@@ -137,14 +153,15 @@ fp2_status fp2_dense_prefill(fp2_plan* plan, const void* q, const void* k_cache,
  * of the dense path (status block, work counter, work order, counting-sort histogram) lives in a device array
  * that is part of the library image: about 0.4 MB on every GPU that loads the library, held until exit.
  *   - Limits: at most 65536 segments and 32 KV heads; larger plans are rejected with FP2_ERR_CAPACITY.
- *     BF16 only, like fp2_dense_prefill.
+ *     BF16 and FP8 plans alike (the dense path of an FP8 plan needs no more scratch than that of a BF16 plan).
  *   - The call allocates and frees nothing.  The first call on a device looks up the array's device address
  *     (cudaGetSymbolAddress, with that device current); that first call should come before any stream
  *     capture.
  *   - All calls on a device share the one array, and it keeps what the previous call left: the entry point
  *     clears the words that must start at zero, on `stream`.  Two calls whose kernels overlap on the GPU
  *     (different streams, no dependency) race on it -- serialise them.
- *   - The status block of this variant is internal; fp2_read_status does not see it.
+ *   - The status block of this variant sits in the same array: fp2_read_status(plan, NULL, ...) reads and clears
+ *     it (bounded waits that ran out, page ids that were skipped), like it does for a caller's workspace.
  * Arguments and results as fp2_dense_prefill, without `workspace`. */
 fp2_status fp2_dense_prefill_static(fp2_plan* plan, const void* q, const void* k_cache, const void* v_cache,
                                     const int32_t* page_table, const int32_t* cu_seqlens_q,
@@ -205,8 +222,9 @@ fp2_status fp2_page_table_from_token_map(fp2_plan* plan, const int32_t* token_to
                                          fp2_stream stream);
 
 /* Synchronises `stream`, reads the status block of `workspace` and clears it.  Returns FP2_ERR_TIMEOUT if a
- * bounded wait expired, FP2_ERR_INVALID_ARG if a list entry had to be clamped, else FP2_OK.  If
- * h_status_words is not NULL it receives the 8 raw int32 words (host memory). */
+ * bounded wait expired, FP2_ERR_INVALID_ARG if a list entry had to be clamped or a page id was out of range, else
+ * FP2_OK.  If h_status_words is not NULL it receives the 8 raw int32 words (host memory).  workspace == NULL
+ * selects the status block of fp2_dense_prefill_static on the plan's device, which must be the current one. */
 fp2_status fp2_read_status(fp2_plan* plan, void* workspace, int32_t* h_status_words, fp2_stream stream);
 
 /* Number of kernels the last stage call on this plan enqueued (host counter). */

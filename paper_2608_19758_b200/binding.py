@@ -18,6 +18,7 @@ STATUS_NAMES = {0: "FP2_OK", 1: "FP2_ERR_INVALID_ARG", 2: "FP2_ERR_UNSUPPORTED",
                 4: "FP2_ERR_CUDA", 5: "FP2_ERR_TIMEOUT"}
 
 EXPORTS = ["fp2_plan_create", "fp2_plan_sizes", "fp2_plan_destroy", "fp2_plan_segment", "fp2_select_blocks",
+           "fp2_pool_blocks",
            "fp2_sparse_prefill", "fp2_dense_prefill", "fp2_dense_prefill_static", "fp2_export_csr",
            "fp2_page_table_from_token_map", "fp2_plan_set_split", "fp2_pool_carry", "fp2_pool_carry_count",
            "fp2_read_status", "fp2_last_launch_count", "fp2_status_string"]
@@ -66,6 +67,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.fp2_select_blocks.argtypes = [C.c_void_p, vp, vp, vp, i32p, i32p, i32p, f32p, f32p, f32p, i64p, i32p, i32p,
                                       vp, C.c_void_p]
     lib.fp2_select_blocks.restype = C.c_int
+    lib.fp2_pool_blocks.argtypes = [C.c_void_p, vp, vp, i32p, i32p, f32p, f32p, vp, C.c_void_p]
+    lib.fp2_pool_blocks.restype = C.c_int
     lib.fp2_sparse_prefill.argtypes = [C.c_void_p, vp, vp, vp, i32p, i32p, i32p, i64p, i32p, i32p, f32p, f32p, f32p,
                                        vp, f32p, vp, C.c_int32, C.c_void_p]
     lib.fp2_sparse_prefill.restype = C.c_int
@@ -181,6 +184,12 @@ def fp2_select_blocks(plan: Plan, q, k_cache, v_cache, page_table, cu_seqlens_q,
                                     _ptr(workspace), _stream(stream)), "fp2_select_blocks")
 
 
+def fp2_pool_blocks(plan: Plan, k_cache, v_cache, page_table, seqlens_k, k_scale, v_scale, workspace, stream=None):
+    """Block-mean pooling alone: the pooled statistics of `workspace` are refreshed, no list is written."""
+    _check(load().fp2_pool_blocks(plan.handle, _ptr(k_cache), _ptr(v_cache), _ptr(page_table), _ptr(seqlens_k),
+                                  _ptr(k_scale), _ptr(v_scale), _ptr(workspace), _stream(stream)), "fp2_pool_blocks")
+
+
 def fp2_sparse_prefill(plan: Plan, q, k_cache, v_cache, page_table, cu_seqlens_q, seqlens_k, seg_offset, seg_count,
                        blk_idx, q_scale, k_scale, v_scale, out, lse, workspace, pooled_valid: bool = True,
                        stream=None):
@@ -269,19 +278,39 @@ class DeviceCase:
         self.seg_offset, self.seg_count, self.blk_idx = self.plan.new_lists(dev)
         self.out = torch.empty(case.total_q, prm["num_q_heads"], prm["head_dim"], dtype=torch.bfloat16, device=dev)
         self.lse = torch.empty(prm["num_q_heads"], case.total_q, dtype=torch.float32, device=dev)
+        # Tests set this: every stage call then first overwrites the buffers it is about to fill (lists with -1,
+        # outputs with NaN), so that a row or an entry the call fails to write cannot pass on an earlier call's values.
+        self.poison = False
+
+    def _poison_lists(self):
+        if self.poison:
+            self.seg_count.fill_(-1)
+            self.blk_idx.fill_(-1)
+
+    def _poison_outputs(self):
+        if self.poison:
+            self.out.fill_(float("nan"))
+            self.lse.fill_(float("nan"))
 
     def select(self):
+        self._poison_lists()
         fp2_select_blocks(self.plan, self.q, self.k_cache, self.v_cache, self.page_table, self.cu_seqlens_q,
                           self.seqlens_k, self.q_scale, self.k_scale, self.v_scale, self.seg_offset, self.seg_count,
                           self.blk_idx, self.workspace)
 
+    def pool(self):
+        fp2_pool_blocks(self.plan, self.k_cache, self.v_cache, self.page_table, self.seqlens_k, self.k_scale,
+                        self.v_scale, self.workspace)
+
     def sparse(self, pooled_valid=True, seg_count=None, blk_idx=None):
+        self._poison_outputs()
         fp2_sparse_prefill(self.plan, self.q, self.k_cache, self.v_cache, self.page_table, self.cu_seqlens_q,
                            self.seqlens_k, self.seg_offset, self.seg_count if seg_count is None else seg_count,
                            self.blk_idx if blk_idx is None else blk_idx, self.q_scale, self.k_scale, self.v_scale,
                            self.out, self.lse, self.workspace, pooled_valid)
 
     def dense(self):
+        self._poison_outputs()
         fp2_dense_prefill(self.plan, self.q, self.k_cache, self.v_cache, self.page_table, self.cu_seqlens_q,
                           self.seqlens_k, self.q_scale, self.k_scale, self.v_scale, self.out, self.lse,
                           self.workspace)

@@ -36,6 +36,8 @@ struct DevParams {
   int32_t fp8;
   int32_t q_tma;     // 1: the group size divides 128, so a packed query tile is a TMA box [128 bytes, g heads, 128 / g tokens]
                      //    (x 2 for BF16); used by the attention kernel (both dtypes) and the BF16 scorer
+  int32_t diag_mma;  // 1: a tile spans at most 32 positions (g >= 4), so the causal mask of a diagonal block can ride
+                     //    on a K = 32 one-hot MMA step in the attention kernel
   float alpha;
   float scale_log2;  // softmax scale * log2(e)
 };

@@ -36,6 +36,7 @@ struct fp2_plan {
   SegInfo* d_segs;
   int32_t* d_blk_off;
   int32_t* d_carry;                 // [3 x num_seqs]: pooled rows carried over from a previous chunk (fp2_pool_carry)
+  int32_t* d_lk;                    // [num_seqs]: KV lengths as given to fp2_plan_create
   std::vector<int32_t> h_blk_off, h_carry;
   bool carry_valid;
   // workspace layout (byte offsets)
@@ -156,15 +157,18 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
     pl->num_sms = prop.multiProcessorCount;
     const size_t seg_bytes = (size_t)align_up((int64_t)sizeof(SegInfo) * (pl->nseg > 0 ? pl->nseg : 1), 256);
     const size_t boff_bytes = (size_t)align_up((int64_t)sizeof(int32_t) * blk_off.size(), 256);
-    const size_t tab_bytes = seg_bytes + boff_bytes + sizeof(int32_t) * 3 * (p->num_seqs > 0 ? p->num_seqs : 1);
+    const size_t carry_bytes = (size_t)align_up((int64_t)sizeof(int32_t) * 3 * (p->num_seqs > 0 ? p->num_seqs : 1), 256);
+    const size_t tab_bytes = seg_bytes + boff_bytes + carry_bytes + sizeof(int32_t) * (p->num_seqs > 0 ? p->num_seqs : 1);
     if (cudaMalloc(&pl->d_table, tab_bytes) != cudaSuccess) { delete pl; return FP2_ERR_CUDA; }
     pl->d_segs = reinterpret_cast<SegInfo*>(pl->d_table);
     pl->d_blk_off = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(pl->d_table) + seg_bytes);
     pl->d_carry = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(pl->d_table) + seg_bytes + boff_bytes);
+    pl->d_lk = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(pl->d_table) + seg_bytes + boff_bytes + carry_bytes);
     if ((pl->nseg > 0 && cudaMemcpy(pl->d_segs, segs.data(), sizeof(SegInfo) * segs.size(),
                                     cudaMemcpyHostToDevice) != cudaSuccess) ||
         cudaMemcpy(pl->d_blk_off, blk_off.data(), sizeof(int32_t) * blk_off.size(), cudaMemcpyHostToDevice) !=
-            cudaSuccess) {
+            cudaSuccess ||
+        cudaMemcpy(pl->d_lk, h_lk, sizeof(int32_t) * p->num_seqs, cudaMemcpyHostToDevice) != cudaSuccess) {
       cudaFree(pl->d_table);
       delete pl;
       return FP2_ERR_CUDA;
@@ -221,6 +225,8 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
   d.num_seqs = p->num_seqs; d.nseg = (int32_t)pl->nseg; d.nblk_tot = (int32_t)nblk_tot; d.total_q = p->total_q;
   d.fp8 = p->dtype == FP2_FP8_E4M3;
   d.q_tma = (128 % g == 0) ? 1 : 0;
+  // positions spanned by a 128-row packed tile: 128 / g when g divides 128, else up to floor((g - 1 + 127) / g) + 1
+  d.diag_mma = ((128 % g == 0) ? 128 / g : (g - 1 + 127) / g + 1) <= 32 ? 1 : 0;
   d.alpha = p->alpha;
   const double sc = p->softmax_scale > 0.f ? (double)p->softmax_scale : 1.0 / sqrt((double)kHeadDim);
   d.scale_log2 = (float)(sc * 1.4426950408889634);
@@ -338,12 +344,14 @@ static fp2_status launch_pool(fp2_plan* pl, const void* k, const void* v, const 
   __nv_bfloat16* khi = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_khi);
   __nv_bfloat16* klo = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_klo);
   __nv_bfloat16* vb = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_vbar);
+  int* status = reinterpret_cast<int*>(ws + pl->ws_status);
+  (void)lk;   // the lengths the kernel uses are the plan's own copy
   if (pl->dev.fp8)
-    pool_kv_kernel<true><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, lk, pl->d_blk_off, ks, vs,
-                                               pl->dev, khi, klo, vb, ws + pl->ws_k8hi, ws + pl->ws_k8lo, carry);
+    pool_kv_kernel<true><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, pl->d_lk, pl->d_blk_off, ks, vs,
+                                               pl->dev, khi, klo, vb, ws + pl->ws_k8hi, ws + pl->ws_k8lo, carry, status);
   else
-    pool_kv_kernel<false><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, lk, pl->d_blk_off, ks, vs,
-                                                pl->dev, khi, klo, vb, nullptr, nullptr, carry);
+    pool_kv_kernel<false><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, pl->d_lk, pl->d_blk_off, ks, vs,
+                                                pl->dev, khi, klo, vb, nullptr, nullptr, carry, status);
   pl->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
@@ -400,11 +408,32 @@ extern "C" fp2_status fp2_select_blocks(fp2_plan* pl, const void* q, const void*
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
 
+// Block-mean pooling alone (the first kernel of stage 1)
+extern "C" fp2_status fp2_pool_blocks(fp2_plan* pl, const void* k, const void* v, const int32_t* pt,
+                                      const int32_t* lk, const float* ks, const float* vs, void* workspace,
+                                      fp2_stream stream) {
+  if (!pl || !k || !v || !pt || !lk || !workspace) return FP2_ERR_INVALID_ARG;
+  if (pl->dev.fp8 && (!ks || !vs)) return FP2_ERR_INVALID_ARG;
+  if (!aligned(k, 16) || !aligned(v, 16) || !aligned(workspace, 1024)) return FP2_ERR_INVALID_ARG;
+  if (pl->device < 0) return FP2_ERR_CUDA;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FP2_ERR_CUDA;
+  if (dev != pl->device) return FP2_ERR_INVALID_ARG;
+  pl->last_launches = 0;
+  return launch_pool(pl, k, v, pt, lk, ks, vs, reinterpret_cast<uint8_t*>(workspace),
+                     reinterpret_cast<cudaStream_t>(stream));
+}
+
 // ------------------------------------------------------------------------------------------------------
 // stage 2 (sparse and dense)
 // ------------------------------------------------------------------------------------------------------
 // Attention: two 256-thread CTAs per SM, each a persistent worker on the shared work counter.  mkb / mkb_lo:
 // pooled keys of the correction chunks (BF16: one BF16 array, mkb_lo unused; FP8: e4m3 hi and lo).
+#ifdef FP2_PROFILE
+static long long* g_prof_ptr = nullptr;
+extern "C" void fp2_debug_set_prof(long long* p) { g_prof_ptr = p; }
+#endif
+
 static void launch_attn(fp2_plan* pl, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mkb,
                         const CUtensorMap& mkb_lo, const CUtensorMap& mvb, const CUtensorMap& mq, const AttnArgs& a,
                         int64_t max_units, cudaStream_t st) {
@@ -459,6 +488,9 @@ static fp2_status run_attention(fp2_plan* pl, const void* q, const void* k, cons
   a.work_counter = reinterpret_cast<int*>(ws + pl->ws_counter);
   a.status = reinterpret_cast<int*>(ws + pl->ws_status);
   a.unit_split = nullptr; a.n_units = nullptr; a.part_o = nullptr; a.part_ml = nullptr;
+#ifdef FP2_PROFILE
+  a.prof = g_prof_ptr;
+#endif
   // a part is never shorter than kMinPartLen iterations (or the requested length): nothing to split when even the
   // longest candidate range (plus its correction chunks) is below one and a half such parts
   const int min_len = pl->split_target > 0 ? pl->split_target : kMinPartLen;
@@ -550,7 +582,7 @@ extern "C" fp2_status fp2_dense_prefill_static(fp2_plan* pl, const void* q, cons
   if (!pl || !q || !k || !v || !pt || !cu || !lk || !out) return FP2_ERR_INVALID_ARG;
   if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out, 16)) return FP2_ERR_INVALID_ARG;
   if (pl->device < 0) return FP2_ERR_CUDA;
-  if (pl->dev.fp8) return FP2_ERR_UNSUPPORTED;
+  if (pl->dev.fp8 && (!qs || !ks || !vs)) return FP2_ERR_INVALID_ARG;
   if (pl->nseg > kStaticMaxSegments || pl->prm.num_kv_heads > kStaticMaxKvHeads) return FP2_ERR_CAPACITY;
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return FP2_ERR_CUDA;
@@ -575,8 +607,9 @@ extern "C" fp2_status fp2_dense_prefill_static(fp2_plan* pl, const void* q, cons
   order_scatter_kernel<<<blocks, 256, 0, st>>>(pl->d_segs, nullptr, nseg, hist, order);
   const int64_t slots = (int64_t)pl->prm.num_pages * pl->prm.page_size;
   CUtensorMap mk, mv;
-  if (!make_map(pl, &mk, k, slots, pl->prm.num_kv_heads, pl->prm.page_size, false) ||
-      !make_map(pl, &mv, v, slots, pl->prm.num_kv_heads, pl->prm.page_size, false))
+  const bool fp8 = pl->dev.fp8 != 0;
+  if (!make_map(pl, &mk, k, slots, pl->prm.num_kv_heads, pl->prm.page_size, fp8) ||
+      !make_map(pl, &mv, v, slots, pl->prm.num_kv_heads, pl->prm.page_size, fp8))
     return FP2_ERR_CUDA;
   AttnArgs a;
   a.q = reinterpret_cast<const uint8_t*>(q);
@@ -592,6 +625,9 @@ extern "C" fp2_status fp2_dense_prefill_static(fp2_plan* pl, const void* q, cons
   a.status = reinterpret_cast<int*>(sw);
   // the dense path stages no pooled chunks: the two pooled-mean maps are never dereferenced
   a.unit_split = nullptr; a.n_units = nullptr; a.part_o = nullptr; a.part_ml = nullptr;
+#ifdef FP2_PROFILE
+  a.prof = nullptr;
+#endif
   CUtensorMap mq = mk;   // unused unless q_tma
   if (pl->dev.q_tma && !make_q_map(pl, &mq, q)) return FP2_ERR_CUDA;
   launch_attn(pl, mk, mv, mk, mk, mv, mq, a, pl->nseg, st);
@@ -709,13 +745,24 @@ extern "C" fp2_status fp2_page_table_from_token_map(fp2_plan* pl, const int32_t*
 }
 
 extern "C" fp2_status fp2_read_status(fp2_plan* pl, void* workspace, int32_t* h_words, fp2_stream stream) {
-  if (!pl || !workspace) return FP2_ERR_INVALID_ARG;
+  if (!pl) return FP2_ERR_INVALID_ARG;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   int32_t w[ST_WORDS];
-  uint8_t* ws = reinterpret_cast<uint8_t*>(workspace);
-  if (cudaMemcpyAsync(w, ws + pl->ws_status, sizeof(w), cudaMemcpyDeviceToHost, st) != cudaSuccess) return FP2_ERR_CUDA;
+  uint8_t* status = nullptr;
+  if (workspace) {
+    status = reinterpret_cast<uint8_t*>(workspace) + pl->ws_status;
+  } else {
+    // no workspace: the status block of fp2_dense_prefill_static on the plan's device (the current one)
+    if (pl->device < 0) return FP2_ERR_CUDA;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return FP2_ERR_CUDA;
+    if (dev != pl->device) return FP2_ERR_INVALID_ARG;
+    fp2_status s = static_scratch_for(dev, &status);
+    if (s != FP2_OK) return s;
+  }
+  if (cudaMemcpyAsync(w, status, sizeof(w), cudaMemcpyDeviceToHost, st) != cudaSuccess) return FP2_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return FP2_ERR_CUDA;
-  if (cudaMemsetAsync(ws + pl->ws_status, 0, sizeof(w), st) != cudaSuccess) return FP2_ERR_CUDA;
+  if (cudaMemsetAsync(status, 0, sizeof(w), st) != cudaSuccess) return FP2_ERR_CUDA;
   if (h_words) memcpy(h_words, w, sizeof(w));
   if (w[ST_TIMEOUT]) return FP2_ERR_TIMEOUT;
   if (w[ST_BAD_LIST]) return FP2_ERR_INVALID_ARG;

@@ -16,6 +16,7 @@
 #include <cuda_fp16.h>
 #include <cuda_fp8.h>
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace fp2 {
 
@@ -49,7 +50,7 @@ template <bool FP8>
 __global__ void __launch_bounds__(256, 4) pool_kv_kernel(const uint8_t* __restrict__ k_cache,
                                                          const uint8_t* __restrict__ v_cache,
                                                          const int32_t* __restrict__ page_table,
-                                                         const int32_t* __restrict__ seqlens_k,
+                                                         const int32_t* __restrict__ plan_lk,  // [ns], the plan's copy
                                                          const int32_t* __restrict__ blk_off,  // [ns+1]
                                                          const float* __restrict__ k_scale,
                                                          const float* __restrict__ v_scale, DevParams P,
@@ -58,7 +59,8 @@ __global__ void __launch_bounds__(256, 4) pool_kv_kernel(const uint8_t* __restri
                                                          __nv_bfloat16* __restrict__ vbar,
                                                          uint8_t* __restrict__ kbar8_hi,
                                                          uint8_t* __restrict__ kbar8_lo,
-                                                         const int32_t* __restrict__ carry) {
+                                                         const int32_t* __restrict__ carry,
+                                                         int* __restrict__ status) {
   constexpr int ROW_BYTES = FP8 ? 128 : 256;
   constexpr int CHUNKS = ROW_BYTES / 16;       // 16-byte chunks per token row
   constexpr int EPC = FP8 ? 16 : 8;            // elements per chunk
@@ -80,7 +82,9 @@ __global__ void __launch_bounds__(256, 4) pool_kv_kernel(const uint8_t* __restri
   // chunked prefill: the means of the first carry[3 b + 2] blocks of this sequence were carried over from the
   // previous chunk's workspace (pool_carry_kernel) and are not computed again
   if (carry != nullptr && J < carry[3 * b + 2]) return;
-  const int Lk = seqlens_k[b];
+  // The length comes from the plan's table (validated on the host when the plan was made), like every other piece
+  // of geometry: a block of the pooled arrays always has between 1 and 128 real tokens.
+  const int Lk = plan_lk[b];
   const int ntok = min(kBlock, Lk - J * kBlock);
   const int chunk = threadIdx.x % CHUNKS, rg = threadIdx.x / CHUNKS;
   const int32_t* pt = page_table + (size_t)b * P.max_pages_per_seq;
@@ -94,8 +98,14 @@ __global__ void __launch_bounds__(256, 4) pool_kv_kernel(const uint8_t* __restri
     dv[ps] = make_uint4(0, 0, 0, 0);   // zero bit patterns add 0 in both encodings
     if (tl < ntok) {
       const int j = J * kBlock + tl;
-      const size_t slot = (size_t)pt[j / P.page_size] * P.page_size + (j % P.page_size);
-      dv[ps] = __ldg(reinterpret_cast<const uint4*>(cache + slot * row_stride + (size_t)h * ROW_BYTES + chunk * 16));
+      const int pid = pt[j / P.page_size];
+      if (pid < 0 || pid >= P.num_pages) {
+        // a page id outside the pool: nothing is read for this token (it counts as zeros) and the call is flagged
+        atomicOr(status + ST_BAD_LIST, 2);
+      } else {
+        const size_t slot = (size_t)pid * P.page_size + (j % P.page_size);
+        dv[ps] = __ldg(reinterpret_cast<const uint4*>(cache + slot * row_stride + (size_t)h * ROW_BYTES + chunk * 16));
+      }
     }
   }
   float acc[EPC];

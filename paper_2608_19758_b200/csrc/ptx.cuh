@@ -170,6 +170,18 @@ __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t saddr, uint32_
   return d;
 }
 
+// Shared-memory matrix descriptor without swizzle, K-major: core matrices of 8 rows x 16 bytes (128 contiguous
+// bytes); lbo_bytes = distance between the two core matrices that make up 32 bytes of K, sbo_bytes = distance
+// between consecutive groups of 8 rows.
+__device__ __forceinline__ uint64_t make_smem_desc_plain(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;   // version
+  return d;
+}
+
 // Instruction descriptor for kind::f16 / kind::f8f6f4, fp32 accumulate, dense.
 //   fmt: f16 kinds 0 = F16, 1 = BF16; f8f6f4 kinds 0 = E4M3, 1 = E5M2.   major: 0 = K, 1 = MN.
 __host__ __device__ constexpr uint32_t make_idesc(int M, int N, int a_fmt, int b_fmt, int a_major, int b_major) {

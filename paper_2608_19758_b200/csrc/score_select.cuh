@@ -228,7 +228,8 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
   uint8_t* sQraw = smem + 2 * 32768;                     // FP8: two raw e4m3 tiles of 16 KB
   uint8_t* sStage = smem + kScoreQSlots * 32768;                    // kScoreStages x 32 KB pieces (kbar_hi or kbar_lo chunk)
   float* sE = reinterpret_cast<float*>(sStage + kScoreStages * 32768);  // per candidate: log2 of its energy
-  float* sC = sE + kMaxBlocks;                                          // [kScoreQBufs][128] per-row multiplier (FP8)
+  float* sC = sE + kMaxBlocks;                                          // [kScoreInfoSlots][128] per-row multiplier (FP8); a slot is
+                                                                        // rewritten only after every consumer has released its descriptor
 
   __shared__ SegInfo info[kScoreInfoSlots];
   __shared__ int info_valid[kScoreInfoSlots];
@@ -355,7 +356,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
         widen_tile_f16(sQraw + (k & 1) * 16384, sQ + qb * 32768, t64, 64);
         const SegInfo& sgk = info[k % kScoreInfoSlots];
         for (int j = t64; j < kTileRows; j += 64)
-          sC[qb * 128 + j] = P.scale_log2 * q_scale[sgk.h * P.group + (sgk.r0 + j) % P.group];
+          sC[(k % kScoreInfoSlots) * 128 + j] = P.scale_log2 * q_scale[sgk.h * P.group + (sgk.r0 + j) % P.group];
       }
       fence_proxy_async();
       mbar_arrive(&q_full[qb]);
@@ -496,8 +497,8 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
         mbar_wait(&acc_full[wg], uc & 1, ctx, 142);
         tc_fence_after();
         float m, sum;
-        if (sg.nrows == kTileRows) score_chunk<FP8, false>(lane_addr, cs, sC + qb * 128, kTileRows, &acc_empty[wg], m, sum);
-        else score_chunk<FP8, true>(lane_addr, cs, sC + qb * 128, sg.nrows, &acc_empty[wg], m, sum);
+        if (sg.nrows == kTileRows) score_chunk<FP8, false>(lane_addr, cs, sC + slot * 128, kTileRows, &acc_empty[wg], m, sum);
+        else score_chunk<FP8, true>(lane_addr, cs, sC + slot * 128, sg.nrows, &acc_empty[wg], m, sum);
         const int J = c * 128 + key;
         if (J < ncand) {
           const float e = m + log2f(sum);

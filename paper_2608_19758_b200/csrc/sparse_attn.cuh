@@ -54,6 +54,7 @@ struct TileInfo {
   int32_t valid;     // 0: no more work
   int32_t T;         // exact iterations (listed blocks)
   int32_t nchunk;    // non-empty correction chunks
+  int32_t ndiag;     // listed blocks J >= J_lo: the first ndiag iterations (the list is traversed backwards)
   int32_t dense;
   int32_t it_begin, it_end;   // this unit's part of the iteration sequence [0, T + nchunk) (Eq. 18); all of it unless split
   int32_t parts;              // parts the segment is split into (1: the unit writes the final output)
@@ -83,6 +84,9 @@ struct AttnArgs {
   const int32_t* n_units;
   float* part_o;
   float2* part_ml;
+#ifdef FP2_PROFILE
+  long long* prof;   // [grid][16] cycle counters of the softmax warpgroup (development builds only)
+#endif
 };
 
 constexpr int kPParts = 4;   // P is handed to the issuer in this many column slices (4 or 8)
@@ -91,7 +95,8 @@ template <bool FP8>
 struct AttnCfg {
   static constexpr int kThreads = 256;
   static constexpr int kCtasPerSm = 2;
-  static constexpr int kSmemBytes = 1024 + 3 * kTileBytes;   // both dtypes: 96 KB of tiles
+  static constexpr int kBiasBytes = 4096;                    // one 128 x 32 e5m2 operand without swizzle
+  static constexpr int kSmemBytes = 1024 + 3 * kTileBytes + 2 * kBiasBytes;   // both dtypes: 96 KB of tiles + the mask operands
   // Registers: two CTAs share the file, 128 per thread at launch; setmaxnreg moves them from the service warps
   // to the softmax warps.  The move waits without bound for registers the CTA does not own, so the sum is
   // checked here and the compiled register count is checked on the host before the first launch.
@@ -194,6 +199,20 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
   uint8_t* sV = sK + kTileBytes;                       // 32 KB, 16-bit
   uint8_t* sVraw = sV + kTileBytes;                    // FP8 only: 16 KB raw e4m3 V tile
   (void)sVraw;
+  // Masks enter the logits through the tensor core: one more k-step S += hot . bias^T (kind::f8f6f4, e5m2 x e5m2,
+  // K = 32), which costs 64 cycles of the tensor pipe instead of a TMEM round trip of the softmax warpgroup.
+  //   sHot [128 rows x 32]: row i holds 57344 (the largest e5m2) in column c(i) and zeros elsewhere, c(i) = the
+  //     row's position minus the tile's first position (Eq. 13: floor((r0 + i) / g) - floor(r0 / g)); written by the
+  //     set-up warps with the query tile.  Group sizes with more than 32 positions per tile (g < 4) use i mod 32.
+  //   sBias [128 columns x 32], written by the producer warp per masked iteration:
+  //     diagonal block: bias[j][c] = -57344 where column j is hidden from position c (j > t0 + c), else 0;
+  //     correction chunk: bias[j][c] = -57344 for every c where block j is not to be corrected (selected, or past
+  //       the fully visible range), else 0 -- the todo mask is the same for all rows.
+  // A hidden logit thus carries -3.3e9 (raw units), which the exponential turns into an exact zero.
+  // Both operands are K-major without swizzle: 8-row x 16-byte core matrices, row r at (r / 8) * 256 + (r % 8) * 16,
+  // bytes 16..31 of the row 128 bytes further.
+  uint8_t* sHot = smem + 3 * kTileBytes;
+  uint8_t* sBias = sHot + AttnCfg<FP8>::kBiasBytes;
 
   __shared__ TileInfo info[2];
   __shared__ uint32_t sel_bits[kMaxBlocks / 32];
@@ -210,6 +229,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
   __shared__ uint64_t p_ready[kPParts];   // slice q (128 / kPParts probabilities of every row) of P (G) is in TMEM
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
+  __shared__ int ndiag_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   WaitCtx ctx{A.status, &abort_flag};
@@ -277,6 +297,8 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           }
           ti.T = T;
           ti.nchunk = 0;
+          ti.ndiag = ti.dense ? min(T, ti.sg.J_hi - ti.sg.J_lo + 1) : 0;
+          ndiag_s = 0;
         } else {
           ti.valid = 0;
         }
@@ -293,13 +315,17 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           for (int w = t64; w < nwords; w += kSetupThreads) sel_bits[w] = 0u;
         named_bar_sync(2, kSetupThreads);
         bool bad = false;
+        int nd = 0;
         for (int k = t64; k < T; k += kSetupThreads) {
           const int J = list[k];
           if (J < 0 || J > sg.J_hi || (k > 0 && list[k - 1] >= J)) bad = true;
           if (corr && J >= 0 && J < sg.J_lo) atomicOr(&sel_bits[J >> 5], 1u << (J & 31));
+          nd += J >= sg.J_lo;
         }
         if (bad) atomicOr(A.status + ST_BAD_LIST, 1);
+        if (nd) atomicAdd(&ndiag_s, nd);
         named_bar_sync(2, kSetupThreads);
+        if (t64 == 0) ti.ndiag = ndiag_s;
         if (corr) {
           const int nch = (sg.J_lo + 127) >> 7;
           for (int c = t64; c < nch; c += kSetupThreads) {
@@ -333,6 +359,20 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       if (!valid) break;
       // Q tile: wait until every S = Q K^T of the previous unit has completed, then overwrite
       if (it >= 1) mbar_wait(&q_empty, (it - 1) & 1, ctx, 202);
+      {   // sHot: rows 2 t64 and 2 t64 + 1
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int row = 2 * t64 + u;
+          const int c = P.diag_mma ? (ti.sg.r0 + row) / g - ti.sg.r0 / g : (row & 31);
+          uint32_t w[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+#pragma unroll
+          for (int k = 0; k < 8; ++k) w[k] = (c >> 2) == k ? 0x7bu << ((c & 3) * 8) : 0u;   // e5m2 57344
+          uint8_t* dst = sHot + (row >> 3) * 256 + (row & 7) * 16;
+          *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(dst + 128) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+        fence_proxy_async();
+      }
       if (P.q_tma) {
         // PackGQA (Eq. 13) with a group size that divides 128: the tile is 128 / g tokens x g heads, one TMA box
         // per 128 bytes of a row (two 64-element halves for BF16, the whole row for e4m3), landing in the swizzled
@@ -381,10 +421,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       const int32_t* pt = A.page_table + (size_t)sg.b * P.max_pages_per_seq;
       // page id of this lane's page of exact iteration i (-1: past the end of the sequence, or not an exact
       // iteration).  Fetched one iteration ahead: list entry -> page-table entry are two dependent global loads.
+      int J_fetched = 0;   // block id of the iteration fetch_pid was last asked for (warp-uniform)
       auto fetch_pid = [&](int i) -> int {
-        if (i >= T || lane >= ppb) return -1;
+        if (i >= T) return -1;
         int J = ti.dense ? sg.J_hi - i : list[T - 1 - i];
         J = max(0, min(J, sg.J_hi));
+        J_fetched = J;
+        if (lane >= ppb) return -1;
         if (J * kBlock + lane * psz >= sg.Lk) return -1;
         int pid = pt[J * ppb + lane];
         if (pid < 0 || pid >= P.num_pages) {
@@ -393,11 +436,39 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         }
         return pid;
       };
+      // hidden columns of a masked iteration -> sBias (see there); row j = lane * 4 + u gets 32 bytes of which the
+      // first nh[u] are -57344 (e5m2 0xfb).  The S = Q K^T that last read sBias has completed (wait 302).
+      auto write_bias = [&](const int (&nh)[4]) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int j = lane * 4 + u;
+          uint32_t w[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const int n = nh[u] - 4 * k;   // hidden bytes in this word
+            w[k] = n >= 4 ? 0xfbfbfbfbu : n <= 0 ? 0u : (0xfbfbfbfbu >> (32 - 8 * n));
+          }
+          uint8_t* dst = sBias + (j >> 3) * 256 + (j & 7) * 16;
+          *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(dst + 128) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+        fence_proxy_async();
+        __syncwarp();
+      };
       int pid_next = fetch_pid(ti.it_begin);
       for (int i = ti.it_begin; i < ti.it_end; ++i, ++G) {
         const int pid = pid_next;
+        const int J_cur = J_fetched;
         pid_next = fetch_pid(i + 1);
         if (G >= 1) mbar_wait(&s_done, (G - 1) & 1, ctx, 302);   // K stage free
+        if (i < ti.ndiag && P.diag_mma) {
+          // diagonal block: column j is hidden from the tile's position c iff J * 128 + j > pre + r0 / g + c
+          const int t0 = sg.pre + sg.r0 / g - J_cur * kBlock;
+          int nh[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) nh[u] = max(0, min(32, lane * 4 + u - t0));
+          write_bias(nh);
+        }
         if (i < T) {
           const int nvalid = __popc(__ballot_sync(0xffffffffu, pid >= 0));
           if constexpr (FP8) {
@@ -429,7 +500,15 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
             }
           }
         } else {
-          const int row0 = sg.blk_off + ti.chunk_id[i - T] * 128;
+          const int cid = ti.chunk_id[i - T];
+          const int row0 = sg.blk_off + cid * 128;
+          {
+            const uint32_t w = ti.todo[cid][lane >> 3];
+            int nh[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) nh[u] = ((w >> ((lane * 4 + u) & 31)) & 1u) ? 0 : 32;
+            write_bias(nh);
+          }
           if (lane == 0) {
             mbar_arrive_expect_tx(&k_full, kTileBytes);
             if constexpr (FP8) {   // e4m3 hi | lo, 16 KB each
@@ -495,6 +574,11 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
               umma_f16_ss(tmem, ad, bd, idesc_qk, ks > 0);
             }
           }
+          if (i >= T || (i < ti.ndiag && P.diag_mma)) {   // masked iteration: the mask as one more k-step (see sBias)
+            constexpr uint32_t idesc_bias = make_idesc(128, 128, 1, 1, 0, 0);   // e5m2 x e5m2
+            umma_f8_ss(tmem, make_smem_desc_plain(smem_u32(sHot), 128, 256),
+                       make_smem_desc_plain(smem_u32(sBias), 128, 256), idesc_bias, 1u);
+          }
           umma_commit(&s_done);
           if (i == i1 - 1) umma_commit(&q_empty);
           // O += P V (G)
@@ -525,9 +609,22 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     uint32_t G = 0, rc = 0;   // rc: exact iterations so far (uses of the raw V slot)
     (void)rc;
     const uint64_t stream_pol = l2_policy_evict_first();   // outputs are written once and not read here
+#ifdef FP2_PROFILE
+    long long pf[16];
+    for (int i = 0; i < 16; ++i) pf[i] = 0;
+    const long long pf_t0 = clock64();
+    long long pf_a, pf_b;
+#define PF_BEGIN() pf_a = clock64()
+#define PF_END(k) (pf_b = clock64(), pf[k] += pf_b - pf_a, pf_a = pf_b)
+#else
+#define PF_BEGIN()
+#define PF_END(k)
+#endif
     for (int it = 0;; ++it) {
       const int slot = it & 1;
+      PF_BEGIN();
       mbar_wait(&info_full[slot], (it >> 1) & 1, ctx, 501);
+      PF_END(0);
       const TileInfo& ti = info[slot];
       if (!ti.valid) break;
       const int T = ti.T;
@@ -543,6 +640,10 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         cs_all *= A.q_scale[ti.sg.h * g + r % g] * A.k_scale[ti.sg.h];
         out_scale = A.v_scale[ti.sg.h];
       }
+      // The mask bias is -3.3e9 in raw units; with FP8 scales so small that this is no longer far below every
+      // visible logit of the row, the warp masks in TMEM as well.
+      bool weak_bias = false;
+      if constexpr (FP8) weak_bias = __any_sync(0xffffffffu, !(cs_all * 3.0e9f > 256.f));
       float m = -INFINITY, l = 0.f;
       // block id of the next exact iteration, fetched one iteration ahead
       const int i0 = ti.it_begin, i1 = ti.it_end;
@@ -557,16 +658,18 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
           int J = dense ? J_hi - i : J_next;
           if (!dense && i + 1 < T) J_next = list[T - 2 - i];
           J = max(0, min(J, J_hi));
-          need_mask = J >= J_lo;
+          need_mask = J >= J_lo && (!P.diag_mma || weak_bias);   // else the causal mask is in the logits already
           tok_lim = pos - J * kBlock;
         } else {
-          const int c = ti.chunk_id[i - T];
-          cm0 = ti.todo[c][0];
-          cm1 = ti.todo[c][1];
-          cm2 = ti.todo[c][2];
-          cm3 = ti.todo[c][3];
-          shift = 7.0f;  // log2(128): one pooled row stands for a full block (Eq. 6)
-          need_mask = true;
+          shift = 7.0f;  // log2(128): one pooled row stands for a full block (Eq. 6); the todo mask is in the logits already
+          if (weak_bias) {
+            const int c = ti.chunk_id[i - T];
+            cm0 = ti.todo[c][0];
+            cm1 = ti.todo[c][1];
+            cm2 = ti.todo[c][2];
+            cm3 = ti.todo[c][3];
+            need_mask = true;
+          }
         }
         if constexpr (FP8) {
           // Exact iteration: widen this iteration's raw e4m3 V tile (exactly) into the F16 V stage before looking
@@ -586,9 +689,15 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
             ++rc;
           }
         }
+        PF_BEGIN();
         mbar_wait(&s_done, G & 1, ctx, 502);
+        PF_END(i == i0 ? 1 : (i < T ? 2 : 3));
+#ifdef FP2_PROFILE
+        pf[i == i0 ? 8 : (i < T ? 9 : 10)] += 1;
+#endif
         tc_fence_after();
         if (need_mask) mask_row(s_addr, tok_lim, cm0, cm1, cm2, cm3);
+        PF_END(4);
         uint32_t x[128];
         const float mx = fmaf(row_load_max(s_addr, x), cs_all, shift);  // cs > 0: scaling commutes with the maximum
         const float m_new = fmaxf(m, mx);
@@ -616,8 +725,10 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(&p_ready[kPParts - 1]);
+        PF_END(5);
       }
       // ------------------------------ epilogue ------------------------------
+      PF_BEGIN();
       const SegInfo& sg = ti.sg;
       const float inv = l > 0.f ? out_scale / l : 0.f;
       const bool have_o = i1 > i0;
@@ -629,6 +740,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         wait_pv(G - 1, 503);   // O += P V of the unit's last iteration
         tc_fence_after();
       }
+      PF_END(6);
       if (ti.parts > 1) {
         // one part of a split segment (Eq. 18): leave (O, m, l) unnormalised for the merge kernel
         float* prow = A.part_o + ((size_t)ti.slot * 128 + row) * 128;
@@ -670,7 +782,13 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
         A.lse[(size_t)head * P.total_q + tok] = (m + log2f(l)) * 0.6931471805599453f;
       tc_fence_before();
       mbar_arrive(&info_empty[slot]);
+      PF_END(7);
     }
+#ifdef FP2_PROFILE
+    pf[15] = clock64() - pf_t0;
+    if (tid == 0 && A.prof)
+      for (int i = 0; i < 16; ++i) A.prof[(size_t)blockIdx.x * 16 + i] = pf[i];
+#endif
   }
   // teardown: on the normal path every barrier has been consumed; after an abort give in-flight copies time
   if (abort_flag) __nanosleep(2000000);

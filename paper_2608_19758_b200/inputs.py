@@ -55,6 +55,8 @@ class CaseSpec:
     alpha: float = 0.1
     use_correction: int = 1
     head_dim: int = HEAD_DIM
+    kv_head_offset: int = 0             # this workload holds KV heads [offset, offset + num_kv_heads) of a larger one
+                                        # (enters the per-head seeds only: a head-sharded rank draws its own heads)
 
     @property
     def group(self) -> int:
@@ -211,7 +213,7 @@ def make_case(spec: CaseSpec) -> Case:
         tok = torch.arange(Lk)
         slots = pages[b][tok // p] * p + tok % p
         for h in range(Hkv):
-            q, k, v = _draw_seq_head(spec, b, h, Lk, pre)
+            q, k, v = _draw_seq_head(spec, b, h + spec.kv_head_offset, Lk, pre)
             qf[int(cu[b]):int(cu[b + 1]), h * g:(h + 1) * g] = q.to(store)
             kf[slots, h] = k.to(store)
             vf[slots, h] = v.to(store)

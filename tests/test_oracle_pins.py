@@ -324,6 +324,57 @@ def test_selection_invariants():
         prev = sel
 
 
+def test_margin_by_hand():
+    """The distance to the threshold that decides which list mismatches are excused: |E_J - alpha max E| divided
+    by alpha max E (the threshold of Eq. 20), worked by hand.  E = [1, 0.1005, 0.0999, 0.05], alpha = 0.1: the
+    threshold is 0.1, so the distances are 0.9 / 0.1, 0.0005 / 0.1, 0.0001 / 0.1 and 0.05 / 0.1.  Dividing by
+    max E instead of the threshold would give a tenth of these; dividing by E_J would give 0.9, ~0.005, ~0.001, 1."""
+    E = np.array([1.0, 0.1005, 0.0999, 0.05])
+    idx, margin = O.select_blocks(E, 0.1, np.zeros(4, dtype=bool))
+    assert idx.tolist() == [0, 1]
+    np.testing.assert_allclose(margin, [9.0, 5e-3, 1e-3, 0.5], rtol=0, atol=1e-12)
+    # forced blocks enter the list but their margin is still their energy's distance to the threshold
+    idx, margin = O.select_blocks(E, 0.1, np.array([False, False, False, True]))
+    assert idx.tolist() == [0, 1, 3]
+    np.testing.assert_allclose(margin, [9.0, 5e-3, 1e-3, 0.5], rtol=0, atol=1e-12)
+    # scale invariance: multiplying every energy by a constant changes neither the list nor the margins
+    idx2, margin2 = O.select_blocks(E * 1024.0, 0.1, np.zeros(4, dtype=bool))
+    assert idx2.tolist() == [0, 1]
+    np.testing.assert_allclose(margin2, margin, rtol=1e-12)
+    # alpha = 1: only the maximum reaches the threshold, and it sits on it
+    idx, margin = O.select_blocks(E, 1.0, np.zeros(4, dtype=bool))
+    assert idx.tolist() == [0]
+    np.testing.assert_allclose(margin, [0.0, 0.8995, 0.9001, 0.95], rtol=0, atol=1e-12)
+
+
+def test_margin_is_zero_exactly_on_the_threshold():
+    """margin_J == 0  <=>  E_J == alpha max E, on exactly representable numbers (powers of two), and the margin
+    of a candidate is the relative perturbation of its energy that would flip its membership."""
+    E = np.array([8.0, 2.0, 1.0, 0.5, 2.0])
+    for alpha, on_thr in ((0.25, [1, 4]), (0.125, [2]), (1.0, [0]), (0.3, [])):
+        idx, margin = O.select_blocks(E, alpha, np.zeros(5, dtype=bool))
+        assert sorted(np.nonzero(margin == 0.0)[0].tolist()) == on_thr
+        assert sorted(np.nonzero(E == alpha * E.max())[0].tolist()) == on_thr
+        assert set(on_thr) <= set(idx.tolist())                   # ">=": equality selects
+    rng = np.random.default_rng(11)
+    E = rng.uniform(0.01, 1.0, 200)
+    alpha = 0.3
+    idx, margin = O.select_blocks(E, alpha, np.zeros(200, dtype=bool))
+    thr = alpha * E.max()
+    kept = set(idx.tolist())
+    for J in range(200):
+        if J == int(np.argmax(E)):
+            continue                                              # moving the maximum moves the threshold itself
+        for sign in (-1.0, 1.0):
+            for f, flips in ((0.5, False), (1.5, True)):
+                Ep = E.copy()
+                Ep[J] = E[J] + sign * f * margin[J] * thr         # move E_J by f x margin x threshold
+                in_now = Ep[J] >= thr
+                moved_across = in_now != (J in kept)
+                toward = (sign > 0) != (J in kept)                # toward the threshold
+                assert moved_across == (flips and toward), (J, sign, f)
+
+
 def test_pooled_means_closed_form():
     B = 8
     x = np.arange(27, dtype=np.float64)[:, None] * np.array([[1.0, -2.0]])
