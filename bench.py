@@ -115,6 +115,12 @@ def physical_gpu_index(local: int):
 
 ORACLE_SAMPLE_SEGMENTS = 512      # the same sample in the cpu_baseline leg and in every step of --impl reference
 
+# Thresholds that put the measured block sparsity of the two 131072-token workloads at the sweep's targets (what the
+# GPU arm's bisection finds); the reference arm, which has no GPU to calibrate with, takes its alpha from here so that
+# both arms time the same workload.  Any other (config, sparsity) falls back to the workload's default alpha.
+CALIBRATED_ALPHA = {(3, 0.5): 1.29e-5, (3, 0.75): 1.52e-4, (3, 0.9): 1.26e-3, (3, 0.95): 4.613e-3, (3, 0.98): 3.42e-2,
+                    (4, 0.5): 1.68e-5, (4, 0.75): 1.93e-4, (4, 0.9): 1.66e-3, (4, 0.95): 6.330e-3, (4, 0.98): 4.53e-2}
+
 
 class OracleSampler:
     """Times the oracle (select + corrected attention with its own lists) for the whole workload from a bounded,
@@ -254,11 +260,12 @@ def main():
     ap.add_argument("--config", type=int, default=3)
     ap.add_argument("--scale-down", type=int, default=1)
     ap.add_argument("--sparsity", type=float, default=0.95)
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "heads"],
+                    help="N > 1: every rank its own workload (weak scaling) or the KV heads of ONE workload (strong)")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-fp8", action="store_true")
-    ap.add_argument("--oracle-segments", type=int, default=1024)
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "fp2":
         args.warmup = 3
@@ -274,12 +281,13 @@ def main():
     if args.impl == "reference":
         if rank != 0:
             return
+        if args.scale_down == 1:
+            spec.alpha = CALIBRATED_ALPHA.get((args.config, round(args.sparsity, 4)), spec.alpha)
         case = inputs.make_case(spec)
-        times, fl = [], 0.0
-        # about 6000 segments over the whole run (a few minutes of host time), at most 1024 per step
-        per_step = max(64, min(1024, 6000 // (args.warmup + args.steps)))
+        smp = OracleSampler(case)
+        times = []
         for i in range(args.warmup + args.steps):
-            est, dt, desc, threads = oracle_sample(case, per_step, seed=i)
+            est, dt = smp.step()
             if i >= args.warmup:
                 times.append(est)
         fl = dense_flops(case)
@@ -288,8 +296,11 @@ def main():
         line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-                "config": {"workload": workload, "note": "each step is a bounded sample of the workload, extrapolated to the whole workload; ms_per_step is that estimate"},
-                "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+                "config": {"workload": workload, "target_sparsity": args.sparsity, "alpha": float(spec.alpha),
+                           "note": "each step times the same bounded sample of the workload and extrapolates it; "
+                                   "ms_per_step is that estimate for the whole workload"},
+                "cpu_baseline": {"value": val, "unit": UNIT, "cores": smp.threads(), "kind": "oracle",
+                                 "sample": smp.describe(float(np.mean(times)))},
                 "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
         print(json.dumps(line))
         return
@@ -311,7 +322,11 @@ def main():
         torch.cuda.synchronize()
 
     from paper_2608_19758_b200 import shard
-    spec = shard.shard_spec(spec, rank, world)   # every rank an independent shard: same shape, its own seed
+    whole_spec = spec
+    if args.shard == "heads" and world > 1:
+        spec = shard.shard_spec_by_heads(spec, rank, world)   # this rank's KV heads of the one workload
+    else:
+        spec = shard.shard_spec(spec, rank, world)            # every rank an independent workload: same shape, own seed
     case = inputs.make_case(spec)
     dc = binding.DeviceCase(case)
     peaks = measured_peaks()
@@ -322,13 +337,10 @@ def main():
         return float(dc.seg_count.sum().item()) / pairs
 
     def set_alpha(alpha):
-        nonlocal dc
         prm = dict(dc.prm); prm["alpha"] = float(alpha)
-        old = dc
         dc.plan.close()
-        dc.plan = binding.Plan(prm, case.cu_seqlens_q.tolist(), case.seqlens_k.tolist())
+        dc.plan = binding.Plan(prm, dc.case.cu_seqlens_q.tolist(), dc.case.seqlens_k.tolist())
         dc.prm = prm
-        return old
 
     def calibrate(target_sparsity):
         """Bisection on log(alpha) to the requested measured block sparsity."""
@@ -377,6 +389,61 @@ def main():
         tot = e[0][0].elapsed_time(e[-1][2])
         return sel, att, tot, launches
 
+    def sparse_without_correction(steps, warmup):
+        """The attention call on the same lists with use_correction = 0 (plain truncation, Eq. 4): what the
+        correction chunks of Eq. 6 cost is the difference to the corrected call."""
+        prm0 = dict(dc.prm); prm0["use_correction"] = 0
+        plan0 = binding.Plan(prm0, dc.case.cu_seqlens_q.tolist(), dc.case.seqlens_k.tolist())
+
+        def fn():
+            binding.fp2_sparse_prefill(plan0, dc.q, dc.k_cache, dc.v_cache, dc.page_table, dc.cu_seqlens_q,
+                                       dc.seqlens_k, dc.seg_offset, dc.seg_count, dc.blk_idx, dc.q_scale, dc.k_scale,
+                                       dc.v_scale, dc.out, dc.lse, dc.workspace, True)
+        t = timed(fn, steps, warmup)
+        plan0.close()
+        return float(np.mean(t))
+
+    def sweep_point(target, steps=3, warmup=1):
+        a, s_ = calibrate(target)
+        sm_, am_, _, _ = step_split(steps, warmup)
+        ex = float(dc.seg_count.sum().item()) * 4.0 * 128 ** 3
+        no_corr = sparse_without_correction(steps, warmup)
+        am = float(np.mean(am_))
+        return {"target_sparsity": target, "alpha": a, "sparsity": s_,
+                "select_ms": float(np.mean(sm_)), "sparse_ms": am,
+                "executed_tflops": ex / (am * 1e-3) / 1e12,
+                "dense_equiv_tflops": dense_flops(dc.case) / ((np.mean(sm_) + am) * 1e-3) / 1e12,
+                "sparse_ms_without_correction": no_corr, "correction_overhead_ms": am - no_corr,
+                "correction_overhead_pct": 100.0 * (am - no_corr) / no_corr}
+
+    def select_rooflines(sel_ms_mean):
+        """Rooflines of the two kernels of the index stage.  Pooling is bandwidth-bound (K and V read once).  The
+        scorer has three candidate bounds: bytes (the query tensor once + the energies' lists), tensor work (the
+        pooled-key contraction, twice for the hi / lo pair of pooled keys) and exponentials (one per tile row and
+        candidate block at 16 per cycle and SM); the largest of the three is its bound."""
+        c = dc.case
+        esz = 1 if c.spec.dtype == "fp8" else 2
+        pool_ms = float(np.mean(timed(dc.pool, 10, 3)))
+        kv_bytes = 2.0 * float(c.seqlens_k.sum().item()) * c.spec.num_kv_heads * 128 * esz
+        score_ms = max(sel_ms_mean - pool_ms, 1e-6)
+        q_bytes = float(c.total_q) * c.spec.num_q_heads * 128 * esz
+        sc_bytes = q_bytes + 4.0 * float(dc.seg_count.sum().item()) + 12.0 * dc.plan.num_segments
+        t_hbm = sc_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+        flops = 2.0 * 128 * 128 * pairs * 2.0
+        t_tensor = flops / (peaks["bf16_tflops"] * 1e12) * 1e3
+        sm_clock = (clocks.get("sm_max_mhz") or 1965.0) * 1e6
+        t_mufu = 128.0 * pairs / (16.0 * 148 * sm_clock) * 1e3
+        bound = max(t_hbm, t_tensor, t_mufu)
+        return {"pool_kv": {"bound": "hbm", "ms": pool_ms, "achieved": kv_bytes / (pool_ms * 1e-3) / 1e9,
+                            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": kv_bytes / (pool_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                            "algorithmic_bytes": kv_bytes},
+                "score_select": {"ms": score_ms, "hbm_gbs": sc_bytes / (score_ms * 1e-3) / 1e9,
+                                 "hbm_frac": sc_bytes / (score_ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                 "bound_ms": {"hbm": t_hbm, "tensor": t_tensor, "mufu": t_mufu},
+                                 "bound": max((("hbm", t_hbm), ("tensor", t_tensor), ("mufu", t_mufu)), key=lambda kv: kv[1])[0],
+                                 "frac": bound / score_ms,
+                                 "note": "ms = select call minus the pooling kernel timed alone; frac = largest of the three bounds / ms"}}
+
     # headline configuration
     alpha, sp = calibrate(args.sparsity)
     sampler = ClockSampler(physical_gpu_index(local))
@@ -387,6 +454,7 @@ def main():
     sel_pairs = float(dc.seg_count.sum().item())
     exec_flops = sel_pairs * 4.0 * 128 * 128 * 128
     ms_step = total_ms / args.steps
+    # whole job: FLOPs of full causal attention on all ranks' data / the slowest rank's step
     value, ms_step_max, _ = shard.aggregate(dist, ms_step, dflops, device="cuda")
     value /= 1e12
     att_mean = float(np.mean(att_ms))
@@ -397,11 +465,14 @@ def main():
         # own dense path
         dense_ms = timed(dc.dense, 2, 1)
         extra["dense"] = {"ms": float(np.mean(dense_ms)), "tflops": dflops / (np.mean(dense_ms) * 1e-3) / 1e12}
+        no_corr = sparse_without_correction(5, 2)
         extra["headline"] = {"alpha": alpha, "sparsity": sp, "select_ms": float(np.mean(sel_ms)),
                              "sparse_ms": att_mean, "select_ms_min": float(np.min(sel_ms)),
                              "sparse_ms_min": float(np.min(att_ms)), "executed_tflops": achieved,
                              "tokens_per_s": case.total_q / (ms_step * 1e-3),
-                             "speedup_vs_own_dense": float(np.mean(dense_ms)) / ms_step}
+                             "speedup_vs_own_dense": float(np.mean(dense_ms)) / ms_step,
+                             "sparse_ms_without_correction": no_corr}
+        extra["select"] = {"roofline": select_rooflines(float(np.min(sel_ms)))}
         # index export of the headline lists (Algorithm 1 line 5): compact CSR of 64-token physical tiles.
         # Algorithmic bytes: the lists read once (4 B per listed block), two int32 written per block, one
         # 56-byte segment record and one count read and one cu entry written per segment.
@@ -410,6 +481,16 @@ def main():
         extra["export_csr"] = {"tile_tokens": 64, "entries": int(2 * sel_pairs), "ms": float(np.mean(exp_ms)),
                                "gbs": exp_bytes / (np.mean(exp_ms) * 1e-3) / 1e9,
                                "note": "3 launches; includes two torch.empty allocations of the helper"}
+        if not args.no_cpu:
+            # the oracle on its bounded sample, and the GPU's lists against the oracle's on those segments
+            smp = OracleSampler(case)
+            smp.wl.p.alpha = alpha
+            est, dt = smp.step()
+            extra["cpu_baseline"] = {"value": dense_flops(case) / est / 1e12, "unit": UNIT, "cores": smp.threads(),
+                                     "kind": "oracle", "sample": smp.describe(est), "measured_s": dt + smp.t_q + smp.t_kv,
+                                     "host_cores": os.cpu_count()}
+            extra["near_threshold_excluded"] = {workload: smp.compare_lists(dc)}
+            del smp
         # KV splitting (Eq. 18) on launches with about as many units as workers: attention calls timed with the
         # split plan on (automatic) and off (the default)
         if not args.no_sweep:
@@ -432,7 +513,7 @@ def main():
             extra["split_kv"] = rows
         # chunked prefill (Sec. 4.3): the last 8K-token chunk of a 128K-token sequence; the index stage with the
         # prefix pooled again against the prefix's pooled means carried over from the previous chunk
-        if not args.no_sweep and args.config == 3 and args.scale_down == 1:
+        if not args.no_sweep and args.config == 3 and args.scale_down == 1 and world == 1:
             import copy
             sp_prev = copy.deepcopy(spec); sp_prev.seqs = [(122880, 114688)]
             sp_last = copy.deepcopy(spec); sp_last.seqs = [(131072, 122880)]
@@ -452,18 +533,9 @@ def main():
             extra["chunked_prefill"] = {"workload": "last 8192-token chunk of 131072 tokens, Hq=32 Hkv=8",
                                         "select_ms_pool_all": t_fresh, "select_ms_with_carry": t_carry,
                                         "blocks_carried": 960, "blocks_pooled": 64}
+            del d_prev, d_last
         if not args.no_sweep:
-            sweep = []
-            for target in (0.5, 0.75, 0.9, 0.95, 0.98):
-                a, s_ = calibrate(target)
-                sm_, am_, tot_, _ = step_split(3, 1)
-                ex = float(dc.seg_count.sum().item()) * 4.0 * 128 ** 3
-                sweep.append({"target_sparsity": target, "alpha": a, "sparsity": s_,
-                              "select_ms": float(np.mean(sm_)), "sparse_ms": float(np.mean(am_)),
-                              "executed_tflops": ex / (np.mean(am_) * 1e-3) / 1e12,
-                              "dense_equiv_tflops": dflops / ((np.mean(sm_) + np.mean(am_)) * 1e-3) / 1e12,
-                              "speedup_vs_own_dense": float(np.mean(dense_ms)) / float(np.mean(sm_) + np.mean(am_))})
-            extra["sweep"] = sweep
+            extra["sweep"] = [sweep_point(t) for t in (0.5, 0.75, 0.9, 0.95, 0.98)]
             calibrate(args.sparsity)
         # end to end through the C ABI from pinned host buffers
         if not args.no_e2e:
@@ -483,36 +555,49 @@ def main():
             extra["e2e"] = {"value": dflops / (np.mean(e2e_ms) * 1e-3) / 1e12, "unit": UNIT,
                             "ms_per_step": float(np.mean(e2e_ms)), "h2d_bytes_per_step": int(h2d),
                             "d2h_bytes_per_step": int(d2h)}
+            del hq, hk, hv, hout
         # the FP8 e4m3 workload (config 4: Hq=28, Hkv=4, per-head scales) at the same target sparsity
-        if not args.no_fp8 and args.config == 3 and args.scale_down == 1:
+        if not args.no_fp8 and args.config == 3 and args.scale_down == 1 and world == 1:
+            fp8_peak = measure_fp8_peak()
             main_dc, main_case = dc, case
             case = inputs.make_case(inputs.config_spec(4))
             dc = binding.DeviceCase(case)
             pairs = dc.plan.idx_capacity
             a8, s8 = calibrate(args.sparsity)
-            sm8, am8, tot8, _ = step_split(3, 2)
+            sm8, am8, tot8, _ = step_split(5, 3)
             d8 = timed(dc.dense, 2, 1)
             fl8 = dense_flops(case)
             ex8 = float(dc.seg_count.sum().item()) * 4.0 * 128 ** 3
-            sweep8 = []
-            if not args.no_sweep:
-                for target in (0.5, 0.75, 0.9, 0.98):
-                    a_, s_ = calibrate(target)
-                    sm_, am_, _, _ = step_split(3, 1)
-                    ex_ = float(dc.seg_count.sum().item()) * 4.0 * 128 ** 3
-                    sweep8.append({"target_sparsity": target, "alpha": a_, "sparsity": s_,
-                                   "select_ms": float(np.mean(sm_)), "sparse_ms": float(np.mean(am_)),
-                                   "executed_tflops": ex_ / (np.mean(am_) * 1e-3) / 1e12,
-                                   "speedup_vs_own_dense": float(np.mean(d8)) / float(np.mean(sm_) + np.mean(am_))})
+            nc8 = sparse_without_correction(5, 2)
+            sel8 = select_rooflines(float(np.min(sm8)))
+            sweep8 = [sweep_point(t) for t in (0.5, 0.75, 0.9, 0.98)] if not args.no_sweep else []
+            if sweep8:
+                calibrate(args.sparsity)
             dc.status()
+            ach8 = ex8 / (np.mean(am8) * 1e-3) / 1e12
+            dense8 = fl8 / (np.mean(d8) * 1e-3) / 1e12
+            pk8 = fp8_peak.get("fp8_tflops")
             extra["fp8"] = {"workload": "config 4: fp8 e4m3 1 seq, 131072 KV tokens, Hq=28 Hkv=4 d=128 page=64",
                             "alpha": a8, "sparsity": s8, "select_ms": float(np.mean(sm8)),
-                            "sparse_ms": float(np.mean(am8)), "executed_tflops": ex8 / (np.mean(am8) * 1e-3) / 1e12,
+                            "sparse_ms": float(np.mean(am8)), "executed_tflops": ach8,
+                            "sparse_ms_without_correction": nc8,
                             "dense_equiv_tflops": fl8 / ((np.mean(sm8) + np.mean(am8)) * 1e-3) / 1e12,
-                            "dense_ms": float(np.mean(d8)), "dense_tflops": fl8 / (np.mean(d8) * 1e-3) / 1e12,
+                            "dense_ms": float(np.mean(d8)), "dense_tflops": dense8,
                             "speedup_vs_own_dense": float(np.mean(d8)) / float(np.mean(sm8) + np.mean(am8)),
-                            "sweep": sweep8,
-                            "note": "S = Q K^T runs as an FP8 MMA on the raw e4m3 tiles, O += P V as an F16 MMA on widened V (16-bit probabilities)"}
+                            "peak_measured": fp8_peak,
+                            "roofline": {"bound": "tensor", "kernel": "sparse_attn_kernel<fp8>", "achieved": ach8,
+                                         "peak": pk8, "unit": "TFLOP/s", "frac": (ach8 / pk8) if pk8 else None,
+                                         "dense_path_frac": (dense8 / pk8) if pk8 else None,
+                                         "frac_of_sustained_peak": (ach8 / fp8_peak["fp8_tflops_sustained"]) if pk8 else None,
+                                         "peak_source": "measured in this run: " + fp8_peak["how"]},
+                            "select_roofline": sel8, "sweep": sweep8,
+                            "note": "executed FLOPs = selected (tile, block) pairs x 4*128^3, whatever arithmetic the kernel spends on them"}
+            if not args.no_cpu:
+                smp = OracleSampler(case, n_segments=128)
+                smp.wl.p.alpha = a8
+                smp.step()
+                extra.setdefault("near_threshold_excluded", {})[extra["fp8"]["workload"]] = smp.compare_lists(dc)
+                del smp
             # the continuous batch (config 5: 16 sequences with cached prefixes, page size 16) at the paper's
             # default threshold, BF16 and FP8
             if not args.no_sweep:
@@ -534,27 +619,33 @@ def main():
                 extra["continuous_batch"] = rows
             dc, case = main_dc, main_case
             pairs = dc.plan.idx_capacity
-        if not args.no_cpu:
-            est, dt, desc, threads = oracle_sample(case, args.oracle_segments)
-            extra["cpu_baseline"] = {"value": dense_flops(case) / est / 1e12, "unit": UNIT, "cores": threads,
-                                     "kind": "oracle", "sample": desc, "measured_s": dt,
-                                     "host_cores": os.cpu_count()}
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
     if rank != 0:
         return
-    # DRAM bytes per attention launch (dram__bytes_read.sum + dram__bytes_write.sum, one ncu pass on the full
-    # workload, profiles/bench_config3_launch_list.md): 3.29 GB read + 1.06 GB written at config 3 / 95 % sparsity,
-    # against 1.07 (Q) + 0.54 (K, V) + 1.07 (O) GB algorithmic: K/V pages are re-read from DRAM about four times
-    # because one KV head's 67 MB working set does not stay resident in L2 next to the streaming Q / O traffic.
-    traffic = 4.35e9 if (args.config == 3 and args.scale_down == 1 and abs(args.sparsity - 0.95) < 1e-6) else None
+    # DRAM bytes per attention launch: a tracked record of one ncu capture on a smaller case of the same kernel,
+    # scaled to this launch by the units (selected blocks and tiles) it processes; null when there is no record.
+    traffic = None
+    rec_path = os.path.join(ROOT, "profiles", "sparse_attn_kernel_dram_traffic.json")
+    if os.path.exists(rec_path):
+        try:
+            rec = json.load(open(rec_path))
+            traffic = rec["dram_bytes_per_selected_pair"] * sel_pairs + rec["dram_bytes_per_tile"] * dc.plan.num_segments
+        except Exception:
+            traffic = None
+    scaling = "strong" if (args.shard == "heads" and world > 1) else "weak"
+    if scaling == "strong":
+        workload = (f"config {args.config}: {whole_spec.dtype} {len(whole_spec.seqs)} seq, "
+                    f"{sum(l for l, _ in whole_spec.seqs)} KV tokens, Hq={whole_spec.num_q_heads} "
+                    f"Hkv={whole_spec.num_kv_heads} d=128 page={whole_spec.page_size}, KV heads split over {world} ranks")
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_step_max, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": ms_step_max, "higher_is_better": True, "scaling": scaling, "vs_baseline": None,
         "dtype": "bf16" if spec.dtype == "bf16" else "fp8_e4m3", "data": "synthetic",
-        "config": {"workload": workload, "target_sparsity": args.sparsity, "l2": "inputs (Q 1.07 GB, K+V 0.54 GB) "
-                   "exceed the 126 MB L2; no flush", "step": "fp2_select_blocks + fp2_sparse_prefill"},
+        "config": {"workload": workload, "target_sparsity": args.sparsity, "alpha": alpha,
+                   "l2": "inputs (Q 1.07 GB, K+V 0.54 GB) exceed the 126 MB L2; no flush",
+                   "step": "fp2_select_blocks + fp2_sparse_prefill", "shard": args.shard},
         "clocks": clocks, "gpu_launches": launches,
         "roofline": {"bound": "tensor", "kernel": "sparse_attn_kernel", "achieved": achieved,
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],

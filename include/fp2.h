@@ -227,6 +227,16 @@ fp2_status fp2_page_table_from_token_map(fp2_plan* plan, const int32_t* token_to
  * selects the status block of fp2_dense_prefill_static on the plan's device, which must be the current one. */
 fp2_status fp2_read_status(fp2_plan* plan, void* workspace, int32_t* h_status_words, fp2_stream stream);
 
+/* (No counterpart in the paper: a self-test of the library's failure handling.)  Every wait inside the kernels --
+ * on a bulk copy, an MMA, another warp -- is bounded: after a cycle budget it gives up, records the fact (status
+ * word 0) and the place (word 1) in the status block, and the CTA leaves the ordinary way, releasing its tensor
+ * memory.  This call proves that mechanism on the device without involving the attention path: it launches one
+ * 64-thread CTA that allocates tensor memory and waits, with a budget of 10^6 cycles (under a millisecond), on a
+ * barrier that nobody ever arrives on.  The kernel returns by itself; the following fp2_read_status on the same
+ * workspace returns FP2_ERR_TIMEOUT with words {1, 901 or 902, ...} and clears the block, and later stage calls on
+ * the same plan and workspace are unaffected.  Nothing is allocated; one kernel on `stream`. */
+fp2_status fp2_selftest_bounded_wait(fp2_plan* plan, void* workspace, fp2_stream stream);
+
 /* Number of kernels the last stage call on this plan enqueued (host counter). */
 int32_t fp2_last_launch_count(const fp2_plan* plan);
 

@@ -21,7 +21,7 @@ EXPORTS = ["fp2_plan_create", "fp2_plan_sizes", "fp2_plan_destroy", "fp2_plan_se
            "fp2_pool_blocks",
            "fp2_sparse_prefill", "fp2_dense_prefill", "fp2_dense_prefill_static", "fp2_export_csr",
            "fp2_page_table_from_token_map", "fp2_plan_set_split", "fp2_pool_carry", "fp2_pool_carry_count",
-           "fp2_read_status", "fp2_last_launch_count", "fp2_status_string"]
+           "fp2_read_status", "fp2_selftest_bounded_wait", "fp2_last_launch_count", "fp2_status_string"]
 
 
 class Fp2Error(RuntimeError):
@@ -88,6 +88,8 @@ def load(build_if_missing: bool = True) -> C.CDLL:
     lib.fp2_pool_carry_count.restype = C.c_int
     lib.fp2_plan_set_split.argtypes = [C.c_void_p, C.c_int32]
     lib.fp2_plan_set_split.restype = C.c_int
+    lib.fp2_selftest_bounded_wait.argtypes = [C.c_void_p, vp, C.c_void_p]
+    lib.fp2_selftest_bounded_wait.restype = C.c_int
     lib.fp2_read_status.argtypes = [C.c_void_p, vp, C.POINTER(C.c_int32), C.c_void_p]
     lib.fp2_read_status.restype = C.c_int
     lib.fp2_last_launch_count.argtypes = [C.c_void_p]
@@ -245,6 +247,11 @@ def fp2_pool_carry(dst: Plan, dst_workspace, src: Plan, src_workspace, src_seq, 
     a = (C.c_int32 * max(len(src_seq), 1))(*src_seq)
     _check(load().fp2_pool_carry(dst.handle, _ptr(dst_workspace), src.handle, _ptr(src_workspace), a,
                                  _stream(stream)), "fp2_pool_carry")
+
+
+def fp2_selftest_bounded_wait(plan: Plan, workspace, stream=None):
+    """Launches the library's bounded-wait probe: a wait that runs out, recorded in the status block of `workspace`."""
+    _check(load().fp2_selftest_bounded_wait(plan.handle, _ptr(workspace), _stream(stream)), "fp2_selftest_bounded_wait")
 
 
 def fp2_read_status(plan: Plan, workspace, stream=None, raise_on_error: bool = True):

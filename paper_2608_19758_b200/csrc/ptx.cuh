@@ -23,6 +23,7 @@ enum : int { ST_TIMEOUT = 0, ST_WHERE = 1, ST_BAD_LIST = 2, ST_WORDS = 8 };
 struct WaitCtx {
   int* status;           // global status block
   volatile int* abort;   // CTA-shared flag: once set, every wait returns at once
+  long long budget = FP2_WAIT_CYCLES;   // cycles one wait may take
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -55,6 +56,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Non-blocking test (try_wait may suspend the thread for a while; a thread that watches two barriers polls with this).
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // Waits until the phase with the given parity has completed.  Bounded: on expiry the status
 // block records the site and the CTA-wide abort flag makes all later waits fall through.
 __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& ctx, int where) {
@@ -68,13 +79,21 @@ __device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, const 
         if (where >= 200 && where < 700) ctx.status[3 + (where / 100 - 2)] = where;
         return;
       }
-      if (clock64() - t0 > FP2_WAIT_CYCLES) {
+      if (clock64() - t0 > ctx.budget) {
         *ctx.abort = 1;
         if (atomicCAS(ctx.status + ST_TIMEOUT, 0, 1) == 0) ctx.status[ST_WHERE] = where;
         return;
       }
     }
   }
+}
+// After an abort: waits (bounded by `cycles`, whatever the abort flag says) until the barrier's phase has completed.
+// Used on the way out of a kernel to let work in flight finish before its resources are released.
+__device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity, long long cycles) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity))
+    if (clock64() - t0 > cycles) return false;
+  return true;
 }
 
 __device__ __forceinline__ bool elect_one() {

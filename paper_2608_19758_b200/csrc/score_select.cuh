@@ -240,6 +240,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
   __shared__ float red[2][8];
   __shared__ int wsum[8];
   __shared__ uint64_t e_full[2], sel_done[2];   // async mode: [tile & 1] energies of the tile are complete / its list is written
+  __shared__ uint64_t drain_bar;                // teardown after an abort: every MMA issued by this CTA has completed
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   WaitCtx ctx{status, &abort_flag};
@@ -273,6 +274,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       mbar_init(&full[i], 1);
       mbar_init(&empty[i], 1);
     }
+    mbar_init(&drain_bar, 1);
     fence_barrier_init();
   }
   if (warp == 9) {
@@ -294,11 +296,11 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       const int slot = k % kScoreInfoSlots, qb = k % kScoreQBufs;
       if (k >= kScoreInfoSlots) mbar_wait(&info_empty[slot], ((k / kScoreInfoSlots) - 1) & 1, ctx, 111);
       const int sgi = seg_of(k);
-      const bool valid = sgi >= 0;
-      if (t64 == 0) {
-        info_valid[slot] = valid;
-        if (valid) info[slot] = segs[sgi];
-      }
+      // after a wait has run out somewhere in this CTA no further tile is started
+      if (t64 == 0) info_valid[slot] = sgi >= 0 && !*ctx.abort;
+      named_bar_sync(2, 64);
+      const bool valid = info_valid[slot] != 0;
+      if (t64 == 0 && valid) info[slot] = segs[sgi];
       named_bar_sync(2, 64);
       if (t64 == 0) mbar_arrive(&info_full[slot]);
       if (!valid) return false;
@@ -325,7 +327,8 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
         const int slot = k % kScoreInfoSlots, qb = k % kScoreQBufs;
         if (k >= kScoreInfoSlots) mbar_wait(&info_empty[slot], ((k / kScoreInfoSlots) - 1) & 1, ctx, 111);
         const int sgi = seg_of(k);
-        const bool valid = sgi >= 0;
+        bool valid = sgi >= 0 && !*ctx.abort;   // after a wait has run out no further tile is started
+        valid = __shfl_sync(0xffffffffu, valid, 0);
         if (t64 == 0) {
           info_valid[slot] = valid;
           if (valid) info[slot] = segs[sgi];
@@ -560,7 +563,13 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       mbar_arrive(&info_empty[slot]);
     }
   }
-  if (abort_flag) __nanosleep(2000000);
+  if (abort_flag) {   // MMAs and bulk copies may still be in flight: let them finish before tensor memory goes
+    if (warp == 9 && lane == 0) {
+      umma_commit(&drain_bar);
+      mbar_wait_drain(&drain_bar, 0, 200000000ll);
+    }
+    __nanosleep(2000000);
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 9) tmem_dealloc(tmem, 256);

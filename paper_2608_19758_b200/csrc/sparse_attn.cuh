@@ -89,6 +89,14 @@ struct AttnArgs {
 #endif
 };
 
+#ifdef FP2_PROFILE
+#define PF_BEGIN() pf_a = clock64()
+#define PF_END(k) (pf_b = clock64(), pf[k] += pf_b - pf_a, pf_a = pf_b)
+#else
+#define PF_BEGIN()
+#define PF_END(k)
+#endif
+
 constexpr int kPParts = 4;   // P is handed to the issuer in this many column slices (4 or 8)
 
 template <bool FP8>
@@ -230,6 +238,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
   __shared__ int ndiag_s;
+  __shared__ uint64_t drain_bar;   // teardown after an abort: every MMA issued by this CTA has completed
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   WaitCtx ctx{A.status, &abort_flag};
@@ -249,6 +258,7 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     mbar_init(&s_done, 1);
     mbar_init(&pv_done[0], 1);
     mbar_init(&pv_done[1], 1);
+    mbar_init(&drain_bar, 1);
     for (int i = 0; i < kPParts; ++i) mbar_init(&p_ready[i], 128);
     fence_barrier_init();
   }
@@ -281,7 +291,9 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       if (t64 == 0) {
         const int w = atomicAdd(A.work_counter, 1);
         const int n_units = A.unit_split ? *A.n_units : P.nseg;
-        if (w < n_units) {
+        // after a wait has run out somewhere in this CTA no further unit is started: the terminating descriptor
+        // makes every role leave its loop the ordinary way
+        if (w < n_units && !*ctx.abort) {
           const int seg = A.order[w];
           const int32_t split = A.unit_split ? A.unit_split[w] : pack_split(0, 1, 0);
           ti.parts = (split >> 8) & 0xff;
@@ -614,11 +626,6 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
     for (int i = 0; i < 16; ++i) pf[i] = 0;
     const long long pf_t0 = clock64();
     long long pf_a, pf_b;
-#define PF_BEGIN() pf_a = clock64()
-#define PF_END(k) (pf_b = clock64(), pf[k] += pf_b - pf_a, pf_a = pf_b)
-#else
-#define PF_BEGIN()
-#define PF_END(k)
 #endif
     for (int it = 0;; ++it) {
       const int slot = it & 1;
@@ -790,8 +797,16 @@ sparse_attn_kernel(const __grid_constant__ CUtensorMap map_k, const __grid_const
       for (int i = 0; i < 16; ++i) A.prof[(size_t)blockIdx.x * 16 + i] = pf[i];
 #endif
   }
-  // teardown: on the normal path every barrier has been consumed; after an abort give in-flight copies time
-  if (abort_flag) __nanosleep(2000000);
+  // teardown: on the normal path every barrier has been consumed and every MMA has completed (the epilogue waited
+  // for the last one).  After an abort MMAs and bulk copies may still be in flight: the issuing thread waits (bounded)
+  // for its MMAs, everyone gives the copies time, and only then is tensor memory released.
+  if (abort_flag) {
+    if (warp == 5 && lane == 0) {
+      umma_commit(&drain_bar);
+      mbar_wait_drain(&drain_bar, 0, 200000000ll);
+    }
+    __nanosleep(2000000);
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 5) tmem_dealloc(tmem, 256);

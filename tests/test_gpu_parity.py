@@ -457,6 +457,30 @@ def test_page_ids_outside_the_pool_are_skipped_and_flagged():
         check_attention(dc, wl, lists, dtype=dtype)
 
 
+def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable():
+    """The library's probe kernel waits, with a budget of a million cycles, on a barrier nobody arrives on.  The wait
+    gives up by itself (nothing hangs, nothing traps): FP2_ERR_TIMEOUT with the recorded site, then ordinary calls
+    on the same plan and workspace are green."""
+    spec = inputs.small_spec(seqs=[(900, 0)], num_q_heads=4, num_kv_heads=2, page_size=16, config_id=88)
+    case, dc, wl = make(spec)
+    dc.select(); dc.sparse(); dc.status()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    binding.fp2_selftest_bounded_wait(dc.plan, dc.workspace)
+    t1.record()
+    code, words = dc.status(raise_on_error=False)
+    assert code == 5, (code, words)                      # FP2_ERR_TIMEOUT
+    assert words[0] == 1 and words[1] in (901, 902), words
+    assert t0.elapsed_time(t1) < 100.0                   # the budget is under a millisecond of cycles
+    code, words = dc.status(raise_on_error=False)        # reading cleared the block
+    assert code == 0 and not any(words)
+    dc.select(); dc.status()
+    check_lists(dc, wl)
+    lists = dc.lists_host()
+    dc.sparse(); dc.status()
+    check_attention(dc, wl, lists)
+
+
 def test_two_runs_are_bit_identical():
     spec = inputs.config_spec(2, scale_down=4)
     case, dc, wl = make(spec)
