@@ -40,7 +40,7 @@ struct fp2_plan {
   std::vector<int32_t> h_blk_off, h_carry;
   bool carry_valid;
   // workspace layout (byte offsets)
-  int64_t ws_status, ws_counter, ws_khi, ws_klo, ws_vbar, ws_k8hi, ws_k8lo, ws_v8, ws_order, ws_hist, ws_bytes;
+  int64_t ws_status, ws_counter, ws_khi, ws_klo, ws_vbar, ws_k8hi, ws_k8lo, ws_order, ws_hist, ws_bytes;
   // KV splitting (Eq. 18): only plans with few segments carry the buffers
   bool split_capable;
   int32_t split_target;   // < 0 off, 0 automatic, > 0 requested iterations per part
@@ -200,7 +200,6 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
   const int64_t pooled8 = p->dtype == FP2_FP8_E4M3 ? align_up(nblk_tot * p->num_kv_heads * kHeadDim, 1024) : 0;
   pl->ws_k8hi = o; o += pooled8;
   pl->ws_k8lo = o; o += pooled8;
-  pl->ws_v8 = o;   o += pooled8;    // pooled values as e4m3 (raw units), the FP8 operand of the correction chunks
   pl->ws_order = o; o += align_up(4 * (pl->nseg > 0 ? pl->nseg : 1), 1024);
   pl->ws_hist = o;  o += align_up(4 * ((int64_t)p->num_kv_heads * kCountBuckets + 1), 1024);
   // KV splitting pays when there are fewer units than a few waves of workers; the unit arrays and the partial
@@ -349,11 +348,10 @@ static fp2_status launch_pool(fp2_plan* pl, const void* k, const void* v, const 
   (void)lk;   // the lengths the kernel uses are the plan's own copy
   if (pl->dev.fp8)
     pool_kv_kernel<true><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, pl->d_lk, pl->d_blk_off, ks, vs,
-                                               pl->dev, khi, klo, vb, ws + pl->ws_k8hi, ws + pl->ws_k8lo, ws + pl->ws_v8, carry,
-                                               status);
+                                               pl->dev, khi, klo, vb, ws + pl->ws_k8hi, ws + pl->ws_k8lo, carry, status);
   else
     pool_kv_kernel<false><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, pl->d_lk, pl->d_blk_off, ks, vs,
-                                                pl->dev, khi, klo, vb, nullptr, nullptr, nullptr, carry, status);
+                                                pl->dev, khi, klo, vb, nullptr, nullptr, carry, status);
   pl->last_launches += 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }
@@ -689,8 +687,7 @@ extern "C" fp2_status fp2_pool_carry(fp2_plan* dst, void* dst_workspace, const f
   const unsigned gy = (unsigned)std::min((max_n + 7) / 8, 1024);
   pool_carry_kernel<<<dim3((unsigned)ns, gy), 256, 0, st>>>(
       dst->d_carry, rb16, rb8, sw + src->ws_khi, sw + src->ws_klo, sw + src->ws_vbar, sw + src->ws_k8hi,
-      sw + src->ws_k8lo, sw + src->ws_v8, dw + dst->ws_khi, dw + dst->ws_klo, dw + dst->ws_vbar, dw + dst->ws_k8hi,
-      dw + dst->ws_k8lo, dw + dst->ws_v8);
+      sw + src->ws_k8lo, dw + dst->ws_khi, dw + dst->ws_klo, dw + dst->ws_vbar, dw + dst->ws_k8hi, dw + dst->ws_k8lo);
   dst->last_launches = 1;
   return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
 }

@@ -59,7 +59,6 @@ __global__ void __launch_bounds__(256, 4) pool_kv_kernel(const uint8_t* __restri
                                                          __nv_bfloat16* __restrict__ vbar,
                                                          uint8_t* __restrict__ kbar8_hi,
                                                          uint8_t* __restrict__ kbar8_lo,
-                                                         uint8_t* __restrict__ vbar8,
                                                          const int32_t* __restrict__ carry,
                                                          int* __restrict__ status) {
   constexpr int ROW_BYTES = FP8 ? 128 : 256;
@@ -141,9 +140,6 @@ __global__ void __launch_bounds__(256, 4) pool_kv_kernel(const uint8_t* __restri
         reinterpret_cast<__half*>(kbar_lo)[o] = __float2half_rn(mean - __half2float(hi16));
       } else {
         reinterpret_cast<__half*>(vbar)[o] = hi16;
-        // the FP8 attention kernel multiplies its e4m3 probabilities with this row in an FP8 MMA: the mean of the
-        // raw values at the precision the values themselves are stored in
-        vbar8[o] = __nv_cvt_float_to_fp8(mean, __NV_SATFINITE, __NV_E4M3);
       }
     } else {
       const __nv_bfloat16 hi16 = __float2bfloat16_rn(mean);
@@ -217,11 +213,9 @@ __global__ void order_scatter_kernel(const SegInfo* __restrict__ segs, const int
 __global__ void pool_carry_kernel(const int32_t* __restrict__ carry, int row_bytes16, int row_bytes8,
                                   const uint8_t* __restrict__ s_khi, const uint8_t* __restrict__ s_klo,
                                   const uint8_t* __restrict__ s_vbar, const uint8_t* __restrict__ s_k8hi,
-                                  const uint8_t* __restrict__ s_k8lo, const uint8_t* __restrict__ s_v8,
-                                  uint8_t* __restrict__ d_khi,
+                                  const uint8_t* __restrict__ s_k8lo, uint8_t* __restrict__ d_khi,
                                   uint8_t* __restrict__ d_klo, uint8_t* __restrict__ d_vbar,
-                                  uint8_t* __restrict__ d_k8hi, uint8_t* __restrict__ d_k8lo,
-                                  uint8_t* __restrict__ d_v8) {
+                                  uint8_t* __restrict__ d_k8hi, uint8_t* __restrict__ d_k8lo) {
   const int b = blockIdx.x;
   const int src0 = carry[3 * b], dst0 = carry[3 * b + 1], n = carry[3 * b + 2];
   for (int j = blockIdx.y * 8; j < n; j += gridDim.y * 8) {
@@ -237,7 +231,6 @@ __global__ void pool_carry_kernel(const int32_t* __restrict__ carry, int row_byt
     copy(s_vbar, d_vbar, row_bytes16);
     copy(s_k8hi, d_k8hi, row_bytes8);
     copy(s_k8lo, d_k8lo, row_bytes8);
-    copy(s_v8, d_v8, row_bytes8);
   }
 }
 
