@@ -36,6 +36,9 @@ struct DevParams {
   int32_t fp8;
   int32_t q_tma;     // 1: the group size divides 128, so a packed query tile is a TMA box [128 bytes, g heads, 128 / g tokens]
                      //    (x 2 for BF16); used by the attention kernel (both dtypes) and the BF16 scorer
+  int32_t q_box_tok; // tokens of the box that holds a packed tile's rows: 128 / g, or floor((g - 1 + 127) / g) + 1 when g does not
+                     // divide 128 (the tile then starts r0 % g rows into the box)
+  int32_t q_raw_tma; // 1: FP8 plans whose box fits the scorer's raw staging slot: the scorer fetches query tiles by TMA
   int32_t diag_mma;  // 1: a tile spans at most 32 positions (g >= 4), so the causal mask of a diagonal block can ride
                      //    on a K = 32 one-hot MMA step in the attention kernel
   float alpha;

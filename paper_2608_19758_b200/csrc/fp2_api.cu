@@ -225,6 +225,8 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
   d.num_seqs = p->num_seqs; d.nseg = (int32_t)pl->nseg; d.nblk_tot = (int32_t)nblk_tot; d.total_q = p->total_q;
   d.fp8 = p->dtype == FP2_FP8_E4M3;
   d.q_tma = (128 % g == 0) ? 1 : 0;
+  d.q_box_tok = (128 % g == 0) ? 128 / g : (g - 1 + 127) / g + 1;
+  d.q_raw_tma = (d.fp8 && g <= 128 && d.q_box_tok <= 256 && g * d.q_box_tok * 128 <= kScoreRawBytes) ? 1 : 0;
   // positions spanned by a 128-row packed tile: 128 / g when g divides 128, else up to floor((g - 1 + 127) / g) + 1
   d.diag_mma = ((128 % g == 0) ? 128 / g : (g - 1 + 127) / g + 1) <= 32 ? 1 : 0;
   d.alpha = p->alpha;
@@ -284,13 +286,13 @@ static bool make_map(fp2_plan* pl, CUtensorMap* m, const void* base, int64_t row
 
 // Packed query tile as a TMA box (see DevParams::q_tma): [128 bytes, g heads, 128 / g tokens] of q [total_q, Hq, 128]
 // -- 64 BF16 elements (the tile takes two boxes) or 128 e4m3 bytes (one box).
-static bool make_q_map(fp2_plan* pl, CUtensorMap* m, const void* q) {
+static bool make_q_map(fp2_plan* pl, CUtensorMap* m, const void* q, int box_tokens = 0) {
   const int g = pl->dev.group;
   const bool fp8 = pl->dev.fp8;
   const cuuint64_t esz = fp8 ? 1 : 2;
   cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)pl->prm.num_q_heads, (cuuint64_t)pl->prm.total_q};
   cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * esz, (cuuint64_t)kHeadDim * esz * pl->prm.num_q_heads};
-  cuuint32_t box[3] = {fp8 ? 128u : 64u, (cuuint32_t)g, (cuuint32_t)(128 / g)};
+  cuuint32_t box[3] = {fp8 ? 128u : 64u, (cuuint32_t)g, (cuuint32_t)(box_tokens > 0 ? box_tokens : 128 / g)};
   cuuint32_t es[3] = {1, 1, 1};
   CUresult r = pl->encode(m, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
                           const_cast<void*>(q), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -394,8 +396,10 @@ extern "C" fp2_status fp2_select_blocks(fp2_plan* pl, const void* q, const void*
   if (!make_map(pl, &mhi, ws + pl->ws_khi, pl->nblk_tot, pl->prm.num_kv_heads, 128, false) ||
       !make_map(pl, &mlo, ws + pl->ws_klo, pl->nblk_tot, pl->prm.num_kv_heads, 128, false))
     return FP2_ERR_CUDA;
-  CUtensorMap mq = mhi;   // unused unless q_tma
-  if (pl->dev.q_tma && !make_q_map(pl, &mq, q)) return FP2_ERR_CUDA;
+  CUtensorMap mq = mhi;   // unused unless the scorer takes its query tiles by TMA
+  if (pl->dev.fp8 ? (pl->dev.q_raw_tma && !make_q_map(pl, &mq, q, pl->dev.q_box_tok))
+                  : (pl->dev.q_tma && !make_q_map(pl, &mq, q)))
+    return FP2_ERR_CUDA;
   int* status = reinterpret_cast<int*>(ws + pl->ws_status);
   const unsigned grid = (unsigned)(pl->nseg < pl->num_sms ? pl->nseg : pl->num_sms);
   if (pl->dev.fp8)
@@ -432,6 +436,7 @@ extern "C" fp2_status fp2_pool_blocks(fp2_plan* pl, const void* k, const void* v
 #ifdef FP2_PROFILE
 static long long* g_prof_ptr = nullptr;
 extern "C" void fp2_debug_set_prof(long long* p) { g_prof_ptr = p; }
+extern "C" void fp2_debug_set_score_prof(long long* p) { cudaMemcpyToSymbol(fp2::g_score_prof, &p, sizeof(p)); }
 #endif
 
 static void launch_attn(fp2_plan* pl, const CUtensorMap& mk, const CUtensorMap& mv, const CUtensorMap& mkb,

@@ -15,10 +15,10 @@
 // widened to F16 (exact) and kbar is an F16 (hi, lo) pair.
 //
 // Roles: warps 0-3 / 4-7 = two consumer warpgroups alternating over chunks (TMEM accumulators 0 / 1); warp 8 = TMA
-// producer of kbar pieces; warp 9 = UMMA issuer; warps 10-11 fetch the next segment and stage its query tile into
-// a free Q buffer, so that the next tile's MMAs start while the current tile is still being exponentiated.
-// Selection: by the consumers together at the end of their tile -- or, when the query tiles come by TMA (BF16,
-// group size divides 128) and warp 10 alone can feed them, by warp 11 beside the scoring of the next tile.
+// producer of kbar pieces; warp 9 = UMMA issuer; warp 10 fetches the next segments and stages their query tiles into
+// free Q buffers (by TMA when the tile is a box -- BF16, group size divides 128 --, else with cp.async, widening FP8
+// to F16), so that the next tile's MMAs start while the current tile is still being exponentiated; warp 11 applies
+// threshold and forced sets and writes the ordered list of tile t beside the scoring of tile t+1.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_fp8.h>
@@ -27,13 +27,18 @@
 
 namespace fp2 {
 
+#ifdef FP2_PROFILE
+__device__ long long* g_score_prof = nullptr;   // development builds: [cta][warpgroup][8] cycle counters
+#endif
 constexpr int kScoreThreads = 384;
 constexpr int kScoreInfoSlots = 4;       // segment descriptors in flight
 constexpr int kScoreQSlots = 3;           // 32 KB query slots.  BF16: three tiles in flight (two loading while one is
                                          // multiplied; one tile in flight per SM cannot cover the HBM latency-
                                          // bandwidth product).  FP8: two F16 tiles + two raw 16 KB staging tiles.
 constexpr int kScoreStages = 3;          // ring of 32 KB pieces: the kbar_hi or the kbar_lo half of a 128-block chunk
-constexpr int kScoreSmemBytes = 1024 /*align*/ + kScoreQSlots * 32768 + kScoreStages * 32768 + kMaxBlocks * 4 + 2048;
+constexpr int kScoreRawBytes = 20480;     // FP8: one raw e4m3 box of a query tile (up to 160 rows of 128 bytes)
+constexpr int kScoreSmemBytes = 1024 /*align*/ + kScoreQSlots * 32768 + kScoreStages * 32768 + kMaxBlocks * 4 + 2048 +
+                                (2 * kScoreRawBytes - 32768);   // the two raw boxes take the third Q slot and 8 KB more
 
 // Query tile -> shared memory in the K-major 128-byte-swizzled layout the UMMA descriptors expect:
 // BF16: two 64-column halves of [128 rows x 128 B]; FP8 is widened to BF16 on the way (exact).
@@ -97,14 +102,15 @@ __device__ __forceinline__ void widen_chunk_f16(const uint4& v, uint8_t* dst, in
 // Loads go in batches of eight ahead of the stores: raw and dst are both shared memory, and a load the compiler
 // cannot prove independent of the previous store waits for it (measured: 1260 cycles per tile with 128 threads
 // against 885 with the loads hoisted).
+// row_off: the tile's first row inside the raw buffer (a TMA box may start a few packed rows before the tile).
 __device__ __forceinline__ void widen_tile_f16(const uint8_t* __restrict__ raw, uint8_t* __restrict__ dst, int t,
-                                               int nthr) {
+                                               int nthr, int row_off = 0) {
   for (int i0 = t; i0 < kTileRows * 8; i0 += 8 * nthr) {
     uint4 v[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       const int i = i0 + u * nthr;
-      if (i < kTileRows * 8) v[u] = *reinterpret_cast<const uint4*>(raw + sw128_offset(i >> 3, i & 7));
+      if (i < kTileRows * 8) v[u] = *reinterpret_cast<const uint4*>(raw + sw128_offset((i >> 3) + row_off, i & 7));
     }
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
@@ -225,8 +231,8 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   constexpr int kScoreQBufs = FP8 ? 2 : 3;
   uint8_t* sQ = smem;                                    // kScoreQBufs x 32 KB query tiles (+ raw staging, FP8)
-  uint8_t* sQraw = smem + 2 * 32768;                     // FP8: two raw e4m3 tiles of 16 KB
-  uint8_t* sStage = smem + kScoreQSlots * 32768;                    // kScoreStages x 32 KB pieces (kbar_hi or kbar_lo chunk)
+  uint8_t* sQraw = smem + 2 * 32768;                     // FP8: two raw e4m3 boxes of kScoreRawBytes
+  uint8_t* sStage = smem + kScoreQSlots * 32768 + (2 * kScoreRawBytes - 32768);   // kScoreStages x 32 KB pieces (kbar_hi or kbar_lo chunk)
   float* sE = reinterpret_cast<float*>(sStage + kScoreStages * 32768);  // per candidate: log2 of its energy
   float* sC = sE + kMaxBlocks;                                          // [kScoreInfoSlots][128] per-row multiplier (FP8); a slot is
                                                                         // rewritten only after every consumer has released its descriptor
@@ -238,8 +244,8 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_flag;
   __shared__ float red[2][8];
-  __shared__ int wsum[8];
-  __shared__ uint64_t e_full[2], sel_done[2];   // async mode: [tile & 1] energies of the tile are complete / its list is written
+  __shared__ uint64_t e_full[2], sel_done[2];   // [tile & 1] energies of the tile are complete / its list is written
+  __shared__ uint64_t raw_full[2];              // FP8, raw boxes by TMA: box k & 1 has landed
   __shared__ uint64_t drain_bar;                // teardown after an abort: every MMA issued by this CTA has completed
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -250,16 +256,16 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
   // t+1.  The energy buffer is used in two halves by tile parity; a tile with more than kMaxBlocks / 2 candidates
   // takes both and waits for its neighbours.  In this mode the two warpgroups also share the chunks by a count
   // that runs across tiles, so a tile with an odd number of chunks leaves neither of them short.
-  const bool async_sel = !FP8 && P.q_tma;
+  const bool q_by_tma = !FP8 && P.q_tma;   // else warp 10 stages the tile with cp.async (and widens FP8 to F16)
 
   if (tid == 0) {
     abort_flag = 0;
     for (int i = 0; i < kScoreInfoSlots; ++i) {
       mbar_init(&info_full[i], 1);
-      mbar_init(&info_empty[i], 2 + 256 + (async_sel ? 1 : 0));   // producer, issuer, consumers (, selection warp)
+      mbar_init(&info_empty[i], 2 + 256 + 1);   // producer, issuer, consumers, selection warp
     }
     for (int i = 0; i < kScoreQBufs; ++i) {
-      mbar_init(&q_full[i], async_sel ? 1 : 64);
+      mbar_init(&q_full[i], q_by_tma ? 1 : 32);
       mbar_init(&q_empty[i], 1);
     }
     for (int i = 0; i < 2; ++i) {
@@ -275,6 +281,8 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       mbar_init(&empty[i], 1);
     }
     mbar_init(&drain_bar, 1);
+    mbar_init(&raw_full[0], 1);
+    mbar_init(&raw_full[1], 1);
     fence_barrier_init();
   }
   if (warp == 9) {
@@ -286,11 +294,11 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
 
-  if (warp == 10 || (warp == 11 && !async_sel)) {
-    // ---------------- set-up (warps 10 and 11; warp 10 alone when the tiles come by TMA): segment k of this CTA is number blockIdx.x + k * gridDim.x in heaviest-first order
+  if (warp == 10) {
+    // ---------------- set-up (warp 10): segment k of this CTA is number blockIdx.x + k * gridDim.x in heaviest-first order
     // (a static round-robin: no atomic on the critical path).  The loop is software-pipelined: the copies of
     // tile k+1 are issued before the copies of tile k are waited for, so two query tiles are in flight.
-    const int t64 = tid - 320;
+    const int t64 = lane;
     auto seg_of = [&](int k) { return P.nseg - 1 - ((int)blockIdx.x + k * (int)gridDim.x); };
     auto issue = [&](int k) -> bool {   // publishes tile k's descriptor and starts its query copies
       const int slot = k % kScoreInfoSlots, qb = k % kScoreQBufs;
@@ -298,25 +306,39 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       const int sgi = seg_of(k);
       // after a wait has run out somewhere in this CTA no further tile is started
       if (t64 == 0) info_valid[slot] = sgi >= 0 && !*ctx.abort;
-      named_bar_sync(2, 64);
+      __syncwarp();
       const bool valid = info_valid[slot] != 0;
       if (t64 == 0 && valid) info[slot] = segs[sgi];
-      named_bar_sync(2, 64);
-      if (t64 == 0) mbar_arrive(&info_full[slot]);
+      __syncwarp();
+      if (t64 == 0) {
+        __threadfence_block();
+        mbar_arrive(&info_full[slot]);
+      }
       if (!valid) return false;
       const SegInfo sg = info[slot];
       if constexpr (FP8) {
-        // raw e4m3 tile into the staging slot (its previous content was widened two tiles ago by these threads)
-        load_q_raw_async(sQraw + (k & 1) * 16384, q, sg, P, t64, 64);
+        // raw e4m3 rows into the staging slot (its previous content was widened two tiles ago by these threads).
+        // Under PackGQA (Eq. 13) the tile's rows are consecutive (token, head) pairs of the KV head's group: the box
+        // [128 bytes, g heads, q_box_tok tokens] that starts at the tile's first token holds them all, in packed
+        // order, the tile's first row sg.r0 % g rows into it.  One TMA copy instead of 1024 address computations.
+        if (P.q_raw_tma) {
+          if (t64 == 0) {
+            mbar_arrive_expect_tx(&raw_full[k & 1], (uint32_t)(P.group * P.q_box_tok * 128));
+            tma_load_3d_hint(sQraw + (k & 1) * kScoreRawBytes, &map_q, &raw_full[k & 1], 0, sg.h * P.group,
+                             sg.q_tok0 + sg.r0 / P.group, l2_policy_evict_first());
+          }
+        } else {
+          load_q_raw_async(sQraw + (k & 1) * kScoreRawBytes, q, sg, P, t64, 32);
+        }
       } else {
         // the Q buffer is free once every MMA of the tile that used it kScoreQBufs tiles ago has completed
         if (k >= kScoreQBufs) mbar_wait(&q_empty[qb], ((k / kScoreQBufs) - 1) & 1, ctx, 112);
-        load_q_tile_async(sQ + qb * 32768, q, sg, P, t64, 64, false);
+        load_q_tile_async(sQ + qb * 32768, q, sg, P, t64, 32, false);
       }
       cp_async_commit();
       return true;
     };
-    if (async_sel) {
+    if (q_by_tma) {
       // Under PackGQA (Eq. 13) packed row r is (token r / g, head r % g): when g divides 128 a tile is 128 / g
       // consecutive tokens x g consecutive heads, i.e. one TMA box per 64-element half, landing in exactly the
       // swizzled layout the MMA reads.  No thread touches the data; the tile's barrier carries the byte count.
@@ -348,26 +370,49 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
         __syncwarp();
       }
     } else {
+#ifdef FP2_PROFILE
+    long long sp[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    long long sa = clock64(), sb;
+    const long long st0 = sa;
+#define STP(k) (sb = clock64(), sp[k] += sb - sa, sa = sb)
+#else
+#define STP(k)
+#endif
     bool have = issue(0);
-    for (int k = 0; have; ++k) {
+    int k = 0;
+    for (; have; ++k) {
+      STP(4);
       const bool next = issue(k + 1);
+      STP(0);
       if (next) cp_async_wait_group<1>(); else cp_async_wait_group<0>();
+      STP(1);
       const int qb = k % kScoreQBufs;
       if constexpr (FP8) {
-        named_bar_sync(2, 64);   // every thread's copies of tile k have landed
+        const SegInfo& sgw = info[k % kScoreInfoSlots];
+        if (P.q_raw_tma) mbar_wait(&raw_full[k & 1], (k >> 1) & 1, ctx, 114);
+        __syncwarp();   // every thread's copies of tile k have landed
         if (k >= kScoreQBufs) mbar_wait(&q_empty[qb], ((k / kScoreQBufs) - 1) & 1, ctx, 113);
-        widen_tile_f16(sQraw + (k & 1) * 16384, sQ + qb * 32768, t64, 64);
+        STP(2);
+        widen_tile_f16(sQraw + (k & 1) * kScoreRawBytes, sQ + qb * 32768, t64, 32, P.q_raw_tma ? sgw.r0 % P.group : 0);
+        STP(3);
         const SegInfo& sgk = info[k % kScoreInfoSlots];
-        for (int j = t64; j < kTileRows; j += 64)
+        for (int j = t64; j < kTileRows; j += 32)
           sC[(k % kScoreInfoSlots) * 128 + j] = P.scale_log2 * q_scale[sgk.h * P.group + (sgk.r0 + j) % P.group];
       }
       fence_proxy_async();
       mbar_arrive(&q_full[qb]);
       have = next;
     }
+#ifdef FP2_PROFILE
+    if (g_score_prof && t64 == 0) {
+      sp[5] = k;
+      sp[7] = clock64() - st0;
+      for (int i = 0; i < 8; ++i) g_score_prof[((size_t)gridDim.x * 2 + blockIdx.x) * 8 + i] = sp[i];
+    }
+#endif
     }
   } else if (warp == 11) {
-    // ---------------- selection warp (async mode): threshold, forced blocks, ordered compaction of tile `it` ----------------
+    // ---------------- selection warp: threshold, forced blocks, ordered compaction of tile `it` ----------------
     for (int it = 0;; ++it) {
       const int slot = it % kScoreInfoSlots, eb = it & 1;
       mbar_wait(&info_full[slot], (it / kScoreInfoSlots) & 1, ctx, 151);
@@ -431,7 +476,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
     // ---------------- UMMA issuer: acc[c & 1] = kbar_hi Q^T + kbar_lo Q^T ----------------
     if (lane == 0) {
       constexpr uint32_t idesc = FP8 ? make_idesc(128, 128, 0, 0, 0, 0) : make_idesc(128, 128, 1, 1, 0, 0);
-      uint32_t pc = 0, ac0 = 0, ac1 = 0, gc0 = 0;   // gc0: chunks of all earlier tiles (async mode), else 0
+      uint32_t pc = 0, ac0 = 0, ac1 = 0, gc0 = 0;   // gc0: chunks of all earlier tiles
       for (int it = 0;; ++it) {
         const int slot = it % kScoreInfoSlots, qb = it % kScoreQBufs;
         mbar_wait(&info_full[slot], (it / kScoreInfoSlots) & 1, ctx, 131);
@@ -463,7 +508,7 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
         }
         umma_commit(&q_empty[qb]);
         mbar_arrive(&info_empty[slot]);
-        if (async_sel) gc0 += nchunks;
+        gc0 += nchunks;
       }
     }
   } else {
@@ -473,14 +518,29 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
     const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + wg * 128;
     const float cs = P.scale_log2;
     uint32_t uc = 0;  // uses of this warpgroup's accumulator
-    uint32_t gc0 = 0;  // chunks of all earlier tiles (async mode), else 0
+    uint32_t gc0 = 0;  // chunks of all earlier tiles
     bool prev_big = false;
+#ifdef FP2_PROFILE
+    long long pf[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const long long pf_t0 = clock64();
+    long long pf_a = pf_t0, pf_b;
+#define SPF(k) (pf_b = clock64(), pf[k] += pf_b - pf_a, pf_a = pf_b)
+#else
+#define SPF(k)
+#endif
     for (int it = 0;; ++it) {
-      const int slot = it % kScoreInfoSlots, qb = it % kScoreQBufs;
+      const int slot = it % kScoreInfoSlots;
+      SPF(3);
       mbar_wait(&info_full[slot], (it / kScoreInfoSlots) & 1, ctx, 141);
+      SPF(0);
+#ifdef FP2_PROFILE
+      if (!info_valid[slot] && g_score_prof && lane == 0 && (warp & 3) == 0) {
+        pf[7] = clock64() - pf_t0;
+        for (int i = 0; i < 8; ++i) g_score_prof[((size_t)blockIdx.x * 2 + wg) * 8 + i] = pf[i];
+      }
+#endif
       if (!info_valid[slot]) break;
       const SegInfo sg = info[slot];
-      const int seg = sg.seg;
       const int ncand = sg.J_hi + 1;
       const int nchunks = (ncand + 127) >> 7;
       // per candidate: log2 of its energy, e_J = m_J + log2(S_J)  (Eq. 1-2 / Eq. 20 in the log domain: the
@@ -488,16 +548,19 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
       float lmax = -INFINITY;
       const int eb = it & 1;
       const bool big = ncand > kMaxBlocks / 2;
-      float* e_out = sE + ((async_sel && !big) ? eb * (kMaxBlocks / 2) : 0);
-      if (async_sel) {
-        // the half of the energy buffer this tile writes must have been read by the selection of tile it-2, and a
-        // tile that takes (or follows one that took) the whole buffer also waits for tile it-1
-        if (it >= 2) mbar_wait(&sel_done[eb], ((it >> 1) - 1) & 1, ctx, 143);
-        if (it >= 1 && (big || prev_big)) mbar_wait(&sel_done[eb ^ 1], ((it - 1) >> 1) & 1, ctx, 144);
-        prev_big = big;
-      }
+      float* e_out = sE + (!big ? eb * (kMaxBlocks / 2) : 0);
+      // the half of the energy buffer this tile writes must have been read by the selection of tile it-2, and a
+      // tile that takes (or follows one that took) the whole buffer also waits for tile it-1
+      if (it >= 2) mbar_wait(&sel_done[eb], ((it >> 1) - 1) & 1, ctx, 143);
+      if (it >= 1 && (big || prev_big)) mbar_wait(&sel_done[eb ^ 1], ((it - 1) >> 1) & 1, ctx, 144);
+      prev_big = big;
       for (int c = (int)((gc0 ^ (uint32_t)wg) & 1u); c < nchunks; c += 2, ++uc) {
+        SPF(3);
         mbar_wait(&acc_full[wg], uc & 1, ctx, 142);
+        SPF(1);
+#ifdef FP2_PROFILE
+        pf[5] += 1;
+#endif
         tc_fence_after();
         float m, sum;
         if (sg.nrows == kTileRows) score_chunk<FP8, false>(lane_addr, cs, sC + slot * 128, kTileRows, &acc_empty[wg], m, sum);
@@ -508,59 +571,16 @@ score_select_kernel(const __grid_constant__ CUtensorMap map_khi, const __grid_co
           e_out[J] = e;
           lmax = fmaxf(lmax, e);
         }
+        SPF(2);
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) lmax = fmaxf(lmax, __shfl_xor_sync(0xffffffffu, lmax, o));
-      if (async_sel) {
-        // hand the tile to the selection warp and go on
-        if (lane == 0) red[eb][warp] = lmax;
-        __syncwarp();
-        mbar_arrive(&e_full[eb]);
-        mbar_arrive(&info_empty[slot]);
-        gc0 += (uint32_t)nchunks;
-        continue;
-      }
-      // ---------------- selection: all 256 consumer threads, three barriers per tile ----------------
-      if (lane == 0) red[0][warp] = lmax;
-      named_bar_sync(1, 256);            // energies and per-warp maxima are visible
-      float maxE = red[0][0];
-#pragma unroll
-      for (int i = 1; i < 8; ++i) maxE = fmaxf(maxE, red[0][i]);
-      // J selected  <=>  E_J >= alpha max E  <=>  e_J >= log2(alpha) + max e   (alpha <= 0 selects everything)
-      const float thr = P.alpha > 0.f ? maxE + log2f(P.alpha) : -INFINITY;
-      const int win_lo = sg.J_lo - P.window_blocks;
-      // warp w owns candidates [w * per, (w + 1) * per), per a multiple of 32: count, exchange, write in order
-      const int per = (((ncand + 7) >> 3) + 31) & ~31;
-      const int beg = warp * per, end = min(beg + per, ncand);
-      int mine = 0;
-      for (int J0 = beg; J0 < end; J0 += 32) {
-        const int J = J0 + lane;
-        const bool keep = J < end && (sE[J] >= thr || J < P.sink_blocks || J >= win_lo);
-        mine += __popc(__ballot_sync(0xffffffffu, keep));
-      }
-      if (lane == 0) wsum[warp] = mine;
-      named_bar_sync(1, 256);
-      int pos = 0, total = 0;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int v = wsum[i];
-        pos += (i < warp) ? v : 0;
-        total += v;
-      }
-      for (int J0 = beg; J0 < end; J0 += 32) {
-        const int J = J0 + lane;
-        const bool keep = J < end && (sE[J] >= thr || J < P.sink_blocks || J >= win_lo);
-        const unsigned bal = __ballot_sync(0xffffffffu, keep);
-        if (keep) blk_idx[sg.off + pos + __popc(bal & ((1u << lane) - 1u))] = J;
-        pos += __popc(bal);
-      }
-      if (tid == 0) {
-        seg_count[seg] = total;
-        seg_offset[seg] = sg.off;
-        if (seg == P.nseg - 1) seg_offset[P.nseg] = sg.off + ncand;
-      }
-      named_bar_sync(1, 256);            // sE, red and wsum are reused by the next tile
+      // hand the tile to the selection warp and go on
+      if (lane == 0) red[eb][warp] = lmax;
+      __syncwarp();
+      mbar_arrive(&e_full[eb]);
       mbar_arrive(&info_empty[slot]);
+      gc0 += (uint32_t)nchunks;
     }
   }
   if (abort_flag) {   // MMAs and bulk copies may still be in flight: let them finish before tensor memory goes
