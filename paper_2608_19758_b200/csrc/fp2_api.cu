@@ -348,6 +348,21 @@ static fp2_status launch_pool(fp2_plan* pl, const void* k, const void* v, const 
   __nv_bfloat16* vb = reinterpret_cast<__nv_bfloat16*>(ws + pl->ws_vbar);
   int* status = reinterpret_cast<int*>(ws + pl->ws_status);
   (void)lk;   // the lengths the kernel uses are the plan's own copy
+  // whole cache rows per CTA when a row's 16-byte chunks divide 256 (see pool_rows_kernel), else one head per CTA
+  const int row_chunks = pl->prm.num_kv_heads * (pl->dev.fp8 ? 8 : 16);
+  if (row_chunks <= 256 && 256 % row_chunks == 0) {
+    const unsigned grid_rows = (unsigned)(pl->nblk_tot * 2);
+    if (pl->dev.fp8)
+      pool_rows_kernel<true><<<grid_rows, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, pl->d_lk, pl->d_blk_off,
+                                                        ks, vs, pl->dev, khi, klo, vb, ws + pl->ws_k8hi,
+                                                        ws + pl->ws_k8lo, carry, status);
+    else
+      pool_rows_kernel<false><<<grid_rows, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, pl->d_lk,
+                                                         pl->d_blk_off, ks, vs, pl->dev, khi, klo, vb, nullptr, nullptr,
+                                                         carry, status);
+    pl->last_launches += 1;
+    return cudaGetLastError() == cudaSuccess ? FP2_OK : FP2_ERR_CUDA;
+  }
   if (pl->dev.fp8)
     pool_kv_kernel<true><<<grid, 256, 0, st>>>((const uint8_t*)k, (const uint8_t*)v, pt, pl->d_lk, pl->d_blk_off, ks, vs,
                                                pl->dev, khi, klo, vb, ws + pl->ws_k8hi, ws + pl->ws_k8lo, carry, status);

@@ -42,6 +42,39 @@ __device__ __forceinline__ void accum16(const uint4& v, float* acc) {
   }
 }
 
+// One pooled mean -> the operand formats the scorer and the correction chunks read (see the head of the file).
+template <bool FP8>
+__device__ __forceinline__ void write_pooled(int which, float mean, size_t o, int h, const float* __restrict__ k_scale,
+                                             __nv_bfloat16* __restrict__ kbar_hi, __nv_bfloat16* __restrict__ kbar_lo,
+                                             __nv_bfloat16* __restrict__ vbar, uint8_t* __restrict__ kbar8_hi,
+                                             uint8_t* __restrict__ kbar8_lo) {
+  if constexpr (FP8) {
+    if (which == 0) {
+      // the attention kernel multiplies raw e4m3 queries with this pair in one FP8 MMA group each
+      const __nv_fp8_storage_t hi8 = __nv_cvt_float_to_fp8(mean, __NV_SATFINITE, __NV_E4M3);
+      const float hi8f = __half2float(__half(__nv_cvt_fp8_to_halfraw(hi8, __NV_E4M3)));
+      kbar8_hi[o] = hi8;
+      kbar8_lo[o] = __nv_cvt_float_to_fp8(mean - hi8f, __NV_SATFINITE, __NV_E4M3);
+      mean *= k_scale[h];
+    }
+    const __half hi16 = __float2half_rn(mean);
+    if (which == 0) {
+      reinterpret_cast<__half*>(kbar_hi)[o] = hi16;
+      reinterpret_cast<__half*>(kbar_lo)[o] = __float2half_rn(mean - __half2float(hi16));
+    } else {
+      reinterpret_cast<__half*>(vbar)[o] = hi16;
+    }
+  } else {
+    const __nv_bfloat16 hi16 = __float2bfloat16_rn(mean);
+    if (which == 0) {
+      kbar_hi[o] = hi16;
+      kbar_lo[o] = __float2bfloat16_rn(mean - __bfloat162float(hi16));
+    } else {
+      vbar[o] = hi16;
+    }
+  }
+}
+
 // 1-D grid of nblk_tot * Hkv * 2 CTAs: (K or V) fastest, then the KV head, then the block, so CTAs that run
 // together read neighbouring pieces of the same token rows.  One CTA pools one operand of one (block, head):
 // 128 token rows of 256 B (BF16) / 128 B (FP8).  256 threads, every load of a thread issued before the first
@@ -121,35 +154,104 @@ __global__ void __launch_bounds__(256, 4) pool_kv_kernel(const uint8_t* __restri
     float s = 0.f;
 #pragma unroll
     for (int r = 0; r < ROWS_PER_PASS; ++r) s += red[r][c];
-    float mean = s / (float)ntok;
     const size_t o = ((size_t)gblk * P.num_kv_heads + h) * kHeadDim + c;
-    if constexpr (FP8) {
-      if (which == 0) {
-        // the attention kernel multiplies raw e4m3 queries with this pair in one FP8 MMA group each
-        const __nv_fp8_storage_t hi8 = __nv_cvt_float_to_fp8(mean, __NV_SATFINITE, __NV_E4M3);
-        const float hi8f = __half2float(__half(__nv_cvt_fp8_to_halfraw(hi8, __NV_E4M3)));
-        kbar8_hi[o] = hi8;
-        kbar8_lo[o] = __nv_cvt_float_to_fp8(mean - hi8f, __NV_SATFINITE, __NV_E4M3);
-        mean *= k_scale[h];
+    write_pooled<FP8>(which, s / (float)ntok, o, h, k_scale, kbar_hi, kbar_lo, vbar, kbar8_hi, kbar8_lo);
+  }
+}
+
+// The same pooling with one CTA per (block, K or V) over ALL KV heads: a token's row of the cache is
+// Hkv x 128 elements contiguous, so the CTA streams 128 whole rows (256 KB for 8 BF16 heads) behind ONE look-up of
+// the block's page ids instead of one dependent look-up per 32 KB.  Used when the row's 16-byte chunks divide 256
+// (Hkv a power of two, at most 16 BF16 / 32 FP8 heads).  Thread t owns chunk t mod C of the row and the tokens
+// t / C, t / C + G, ... (G = 256 / C token groups): four 16-byte loads in flight per thread and batch, four CTAs per
+// SM, fp32 accumulation, one shared-memory reduction over the G groups.  Page sizes are powers of two, so the slot
+// of a token takes a shift and a mask (a division per load made the kernel ALU-bound: 143 -> 110 us at 128K).
+// Measured at 131072 tokens, 8 BF16 heads: 93 us for 537 MB = 5.8 TB/s; a bare streaming read reaches 6.8 TB/s.
+template <bool FP8>
+__global__ void __launch_bounds__(256, 4) pool_rows_kernel(const uint8_t* __restrict__ k_cache,
+                                                           const uint8_t* __restrict__ v_cache,
+                                                           const int32_t* __restrict__ page_table,
+                                                           const int32_t* __restrict__ plan_lk,
+                                                           const int32_t* __restrict__ blk_off,
+                                                           const float* __restrict__ k_scale,
+                                                           const float* __restrict__ v_scale, DevParams P,
+                                                           __nv_bfloat16* __restrict__ kbar_hi,
+                                                           __nv_bfloat16* __restrict__ kbar_lo,
+                                                           __nv_bfloat16* __restrict__ vbar,
+                                                           uint8_t* __restrict__ kbar8_hi,
+                                                           uint8_t* __restrict__ kbar8_lo,
+                                                           const int32_t* __restrict__ carry,
+                                                           int* __restrict__ status) {
+  constexpr int CH = FP8 ? 8 : 16;             // 16-byte chunks per head row
+  constexpr int EPC = FP8 ? 16 : 8;            // elements per chunk
+  constexpr int BATCH = 4;                     // loads in flight per thread; four CTAs per SM overlap each other's set-up and reduction
+  __shared__ float red[256 * EPC];             // [token group][chunk][element]
+  __shared__ int32_t pids[kBlock / 8];         // page ids of the block (page size >= 8)
+
+  const int which = blockIdx.x & 1;            // 0: K, 1: V
+  const int gblk = blockIdx.x >> 1;
+  int lo = 0, hi = P.num_seqs;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (blk_off[mid] <= gblk) lo = mid; else hi = mid;
+  }
+  const int b = lo, J = gblk - blk_off[b];
+  if (carry != nullptr && J < carry[3 * b + 2]) return;   // carried over from the previous chunk (pool_carry_kernel)
+  const int Lk = plan_lk[b];
+  const int ntok = min(kBlock, Lk - J * kBlock);
+  const int psz = P.page_size, ppb = P.pages_per_block;
+  const int psz_log2 = 31 - __clz(psz);        // page sizes are powers of two: shifts and masks, no divisions per load
+  if ((int)threadIdx.x < ppb) {
+    int pid = -1;
+    if ((int)threadIdx.x * psz < ntok) {
+      pid = page_table[(size_t)b * P.max_pages_per_seq + J * ppb + threadIdx.x];
+      if (pid < 0 || pid >= P.num_pages) {   // outside the pool: its tokens count as zeros, the call is flagged
+        atomicOr(status + ST_BAD_LIST, 2);
+        pid = -1;
       }
     }
-    if constexpr (FP8) {
-      const __half hi16 = __float2half_rn(mean);
-      if (which == 0) {
-        reinterpret_cast<__half*>(kbar_hi)[o] = hi16;
-        reinterpret_cast<__half*>(kbar_lo)[o] = __float2half_rn(mean - __half2float(hi16));
-      } else {
-        reinterpret_cast<__half*>(vbar)[o] = hi16;
-      }
-    } else {
-      const __nv_bfloat16 hi16 = __float2bfloat16_rn(mean);
-      if (which == 0) {
-        kbar_hi[o] = hi16;
-        kbar_lo[o] = __float2bfloat16_rn(mean - __bfloat162float(hi16));
-      } else {
-        vbar[o] = hi16;
-      }
+    pids[threadIdx.x] = pid;
+  }
+  __syncthreads();
+
+  const int C = P.num_kv_heads * CH;           // chunks per token row; divides 256
+  const int G = 256 / C;
+  const int chunk = threadIdx.x % C, tg = threadIdx.x / C;
+  const int per = kBlock / G;                  // tokens of this thread
+  const size_t row_bytes = (size_t)C * 16;
+  const uint8_t* cache = which ? v_cache : k_cache;
+  float acc[EPC];
+#pragma unroll
+  for (int i = 0; i < EPC; ++i) acc[i] = 0.f;
+  for (int i0 = 0; i0 < per; i0 += BATCH) {
+    // every load of the batch is issued unconditionally (a token that is not there reads the start of the cache
+    // instead and is replaced by zeros afterwards), so that all of them are in flight before the first use
+    uint4 dv[BATCH];
+    bool ok[BATCH];
+#pragma unroll
+    for (int u = 0; u < BATCH; ++u) {
+      const int tl = tg + (i0 + u) * G;        // consecutive token groups interleave: the CTA reads G rows at a time
+      const int pid = pids[min(tl, kBlock - 1) >> psz_log2];
+      ok[u] = i0 + u < per && tl < ntok && pid >= 0;
+      const size_t off = ok[u] ? (((size_t)pid << psz_log2) + (size_t)(tl & (psz - 1))) * row_bytes + chunk * 16 : 0;
+      dv[u] = __ldg(reinterpret_cast<const uint4*>(cache + off));
     }
+#pragma unroll
+    for (int u = 0; u < BATCH; ++u) {
+      if (!ok[u]) dv[u] = make_uint4(0, 0, 0, 0);   // zero bit patterns add 0 in both encodings
+      accum16<FP8>(dv[u], acc);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < EPC; ++i) red[(tg * C + chunk) * EPC + i] = acc[i];
+  __syncthreads();
+  const int nout = C * EPC;                    // Hkv x 128 means
+  for (int o = threadIdx.x; o < nout; o += 256) {
+    float sum = 0.f;
+    for (int r = 0; r < G; ++r) sum += red[r * nout + o];
+    const int h = o / kHeadDim;
+    write_pooled<FP8>(which, sum / (float)ntok, (size_t)gblk * nout + o, h, k_scale, kbar_hi, kbar_lo, vbar, kbar8_hi,
+                      kbar8_lo);
   }
 }
 
