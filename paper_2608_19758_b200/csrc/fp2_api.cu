@@ -14,6 +14,7 @@
 #include "common.cuh"
 #include "pool_kv.cuh"
 #include "score_select.cuh"
+#include "score_pair.cuh"
 #include "sparse_attn.cuh"
 #include "index_export.cuh"
 
@@ -37,6 +38,8 @@ struct fp2_plan {
   int32_t* d_blk_off;
   int32_t* d_carry;                 // [3 x num_seqs]: pooled rows carried over from a previous chunk (fp2_pool_carry)
   int32_t* d_lk;                    // [num_seqs]: KV lengths as given to fp2_plan_create
+  int2* d_units;                    // scorer work units of BF16 plans with TMA query tiles: (segment, second segment or -1)
+  int32_t nunits;
   std::vector<int32_t> h_blk_off, h_carry;
   bool carry_valid;
   // workspace layout (byte offsets)
@@ -144,6 +147,36 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
   pl->carry_valid = false;
   pl->d_carry = nullptr;
 
+  // Scorer work units (score_pair_kernel): adjacent tiles (t-1, t) of one (sequence, KV head) share their candidate
+  // blocks, so they are scored together when the later one has at most kPairMaxCand candidates; heaviest first
+  // (descending segment index, like the single-tile scorer's order).
+  std::vector<int2> units;
+  {
+    int64_t tile_off2 = 0;
+    std::vector<int64_t> toff((size_t)p->num_seqs), ntiles((size_t)p->num_seqs);
+    for (int b = 0; b < p->num_seqs; ++b) {
+      const int lq = h_cu[b + 1] - h_cu[b];
+      ntiles[(size_t)b] = ((int64_t)g * lq + kTileRows - 1) / kTileRows;
+      toff[(size_t)b] = tile_off2;
+      tile_off2 += ntiles[(size_t)b];
+    }
+    for (int b = p->num_seqs - 1; b >= 0; --b)
+      for (int h = p->num_kv_heads - 1; h >= 0; --h) {
+        const int64_t base = p->num_kv_heads * toff[(size_t)b] + (int64_t)h * ntiles[(size_t)b];
+        for (int64_t t = ntiles[(size_t)b] - 1; t >= 0;) {
+          if (t >= 1 && segs[(size_t)(base + t)].J_hi + 1 <= kPairMaxCand) {
+            units.push_back(make_int2((int)(base + t - 1), (int)(base + t)));
+            t -= 2;
+          } else {
+            units.push_back(make_int2((int)(base + t), -1));
+            t -= 1;
+          }
+        }
+      }
+  }
+  pl->nunits = (int32_t)units.size();
+  pl->d_units = nullptr;
+
   // Device part.  Without a usable CUDA device the plan is still returned (sizes and the segment table can be
   // queried), but every stage call on it fails with FP2_ERR_CUDA.
   pl->device = -1;
@@ -158,17 +191,21 @@ extern "C" fp2_status fp2_plan_create(const fp2_params* p, const int32_t* h_cu, 
     const size_t seg_bytes = (size_t)align_up((int64_t)sizeof(SegInfo) * (pl->nseg > 0 ? pl->nseg : 1), 256);
     const size_t boff_bytes = (size_t)align_up((int64_t)sizeof(int32_t) * blk_off.size(), 256);
     const size_t carry_bytes = (size_t)align_up((int64_t)sizeof(int32_t) * 3 * (p->num_seqs > 0 ? p->num_seqs : 1), 256);
-    const size_t tab_bytes = seg_bytes + boff_bytes + carry_bytes + sizeof(int32_t) * (p->num_seqs > 0 ? p->num_seqs : 1);
+    const size_t lk_bytes = (size_t)align_up((int64_t)sizeof(int32_t) * (p->num_seqs > 0 ? p->num_seqs : 1), 256);
+    const size_t tab_bytes = seg_bytes + boff_bytes + carry_bytes + lk_bytes + sizeof(int2) * (units.size() + 1);
     if (cudaMalloc(&pl->d_table, tab_bytes) != cudaSuccess) { delete pl; return FP2_ERR_CUDA; }
     pl->d_segs = reinterpret_cast<SegInfo*>(pl->d_table);
     pl->d_blk_off = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(pl->d_table) + seg_bytes);
     pl->d_carry = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(pl->d_table) + seg_bytes + boff_bytes);
     pl->d_lk = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(pl->d_table) + seg_bytes + boff_bytes + carry_bytes);
+    pl->d_units = reinterpret_cast<int2*>(reinterpret_cast<uint8_t*>(pl->d_table) + seg_bytes + boff_bytes + carry_bytes + lk_bytes);
     if ((pl->nseg > 0 && cudaMemcpy(pl->d_segs, segs.data(), sizeof(SegInfo) * segs.size(),
                                     cudaMemcpyHostToDevice) != cudaSuccess) ||
         cudaMemcpy(pl->d_blk_off, blk_off.data(), sizeof(int32_t) * blk_off.size(), cudaMemcpyHostToDevice) !=
             cudaSuccess ||
-        cudaMemcpy(pl->d_lk, h_lk, sizeof(int32_t) * p->num_seqs, cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaMemcpy(pl->d_lk, h_lk, sizeof(int32_t) * p->num_seqs, cudaMemcpyHostToDevice) != cudaSuccess ||
+        (!units.empty() && cudaMemcpy(pl->d_units, units.data(), sizeof(int2) * units.size(), cudaMemcpyHostToDevice) !=
+                               cudaSuccess)) {
       cudaFree(pl->d_table);
       delete pl;
       return FP2_ERR_CUDA;
@@ -303,7 +340,9 @@ static bool make_q_map(fp2_plan* pl, CUtensorMap* m, const void* q, int box_toke
 
 static fp2_status set_attrs(fp2_plan* pl) {
   if (pl->attrs_set) return FP2_OK;
-  if (cudaFuncSetAttribute(score_select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (cudaFuncSetAttribute(score_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemBytes) !=
+          cudaSuccess ||
+      cudaFuncSetAttribute(score_select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kScoreSmemBytes) != cudaSuccess ||
       cudaFuncSetAttribute(score_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kScoreSmemBytes) != cudaSuccess ||
@@ -420,7 +459,13 @@ extern "C" fp2_status fp2_select_blocks(fp2_plan* pl, const void* q, const void*
   if (pl->dev.fp8)
     score_select_kernel<true><<<grid, kScoreThreads, kScoreSmemBytes, st>>>(
         mhi, mlo, mq, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, status);
-  else
+  else if (pl->dev.q_tma) {
+    // BF16 tiles that are TMA boxes: pairs of adjacent tiles per pooled-key chunk.  The pair kernel takes the pooled
+    // keys in pieces of 64 elements x 128 keys, which is the box of mhi / mlo already.
+    const unsigned grid_pairs = (unsigned)(pl->nunits < pl->num_sms ? pl->nunits : pl->num_sms);
+    score_pair_kernel<<<grid_pairs, kPairThreads, kPairSmemBytes, st>>>(mhi, mlo, mq, pl->d_segs, pl->d_units, pl->nunits,
+                                                                        pl->dev, seg_offset, seg_count, blk_idx, status);
+  } else
     score_select_kernel<false><<<grid, kScoreThreads, kScoreSmemBytes, st>>>(
         mhi, mlo, mq, (const uint8_t*)q, pl->d_segs, qs, pl->dev, seg_offset, seg_count, blk_idx, status);
   pl->last_launches += 1;
