@@ -335,6 +335,27 @@ def test_tiles_with_more_candidates_than_half_the_energy_buffer():
     check_attention(dc, wl, lists, dtype=spec.dtype)
 
 
+def test_scorer_units_pairs_and_singles_of_every_size():
+    """The BF16 scorer takes adjacent tiles of a KV head in pairs when the later tile has at most 1024 candidate
+    blocks, else one by one (a tile with up to 2048 candidates in its unit's half of the energy buffer, beyond that
+    in the whole buffer).  One batch with all three kinds, odd tile counts (a pair cannot straddle two heads or
+    sequences) and a ragged last tile; twice, so that the second run meets whatever the first left behind."""
+    spec = inputs.small_spec(seqs=[(900, 0), (140000 + 1100, 140000), (1300, 300), (266240 + 700, 266240), (385, 0)],
+                             num_q_heads=2, num_kv_heads=2, page_size=64, config_id=62)
+    spec.alpha = 0.05
+    case, dc, wl = make(spec)
+    kinds = {(s.J_hi + 1 > 2048) + (s.J_hi + 1 > 1024) for s in wl.segs}
+    assert kinds == {0, 1, 2}
+    for _ in range(2):
+        dc.select()
+        dc.status()
+        check_lists(dc, wl)
+    lists = dc.lists_host()
+    dc.sparse()
+    dc.status()
+    check_attention(dc, wl, lists, dtype=spec.dtype)
+
+
 @pytest.mark.parametrize("alpha", [0.0, 2.0, 1.0])
 def test_alpha_extremes(alpha):
     spec = inputs.small_spec(seqs=[(2000, 0)], num_q_heads=4, num_kv_heads=1, page_size=64, config_id=81, sink=False)
