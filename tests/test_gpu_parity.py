@@ -23,8 +23,10 @@ NEAR_BAND = 1e-3
 NEAR_SEEN = {}      # test id -> (excluded near-threshold mismatches, candidate pairs compared)
 
 
-def make(spec, **over):
+def make(spec, edit_case=None, **over):
     case = inputs.make_case(spec)
+    if edit_case is not None:
+        edit_case(case)   # e.g. other per-head scales: still a valid input, the oracle sees the same arrays
     dc = binding.DeviceCase(case, **over)
     dc.poison = True    # every stage call first overwrites what it is about to fill (lists -1, outputs NaN)
     prm = dict(case.params())
@@ -79,8 +81,8 @@ def check_attention(dc, wl, lists, seg_ids=None, dense=False, dtype="bf16"):
     return err_o, err_l
 
 
-def full_pipeline(spec, dense=True, **over):
-    case, dc, wl = make(spec, **over)
+def full_pipeline(spec, dense=True, edit_case=None, **over):
+    case, dc, wl = make(spec, edit_case=edit_case, **over)
     dc.select()
     dc.status()
     check_lists(dc, wl)
@@ -262,6 +264,25 @@ def test_fp8_without_sink_and_heavy_pruning():
     spec.alpha = 0.5
     case, dc, wl = full_pipeline(spec, dense=False)
     assert int(dc.seg_count.sum()) < dc.plan.idx_capacity / 2
+
+
+@pytest.mark.parametrize("g,hkv,seqs", [
+    (4, 2, [(1500, 300), (700, 0)]),
+    (7, 1, [(1000, 0), (300, 100)]),
+])
+def test_fp8_query_scales_far_apart_within_a_group(g, hkv, seqs):
+    """The heads of a group with query scales up to 30x apart (Eq. 15 gives every head its own): the scorer's
+    reference maximum is then the exact one instead of the bound it uses for scales within a factor of two, and a
+    packed tile's rows carry very different logit ranges through both kernels."""
+    spec = inputs.small_spec(seqs=seqs, num_q_heads=g * hkv, num_kv_heads=hkv, page_size=16, dtype="fp8",
+                             config_id=60 + g)
+    spec.alpha = 0.1
+
+    def spread(case):
+        case.q_scale[1::2] *= 6.0
+        case.q_scale[2::3] *= 0.2
+
+    full_pipeline(spec, edit_case=spread)
 
 
 def test_config4_relative_at_16k():
